@@ -1,0 +1,153 @@
+/*
+ * allocmoe.h -- C ABI of the budget-constrained MoE layer forward (Alloc-MoE hot path)
+ * for NVIDIA B200 (sm_100a).
+ *
+ * The layer (paper Sec. 3.1 and 3.3):
+ *   Eq. 1   scores = Softmax(x . W_gate) over all N experts, Top-K_orig kept per token
+ *   Alloc-T (Sec. 3.3, procedure paragraph; the 0/1 programme of Eq. 8-10): every token keeps
+ *           its Top-K_base experts; the other K_orig-K_base scores of ALL tokens are pooled and
+ *           the globally largest  budget - K_base*T  of them are kept
+ *   Eq. 2   y_t = sum over kept (t,i) of score[t,i] * E_i(x_t)   (+ shared experts)
+ *
+ * Conventions for every entry point
+ *   - Every pointer marked "device" is device memory owned by the caller, 16-byte aligned,
+ *     valid until the stream has run the call.  The library allocates no device memory,
+ *     never synchronises and launches only on `stream` (a cudaStream_t passed as void*).
+ *   - bf16 tensors are passed as `const uint16_t*` (raw bfloat16 bits), row-major, last index
+ *     contiguous.
+ *   - `budget` is the layer's TOTAL activation count  T*K_l  (Sec. 3.1, "Expert Activation
+ *     Budget"), so fractional per-token averages need no rounding rule.  It must satisfy
+ *     K_base*T <= budget <= K_orig*T  (below: Eq. 10 is infeasible; above: the candidate
+ *     set is exhausted); anything else returns MOE_ERR_BUDGET.
+ *   - Host-checkable errors return a status before anything is launched and leave outputs
+ *     untouched.  Conditions only the device can see (a non-finite or negative score, kept
+ *     counts that do not add up to `budget`, a bounded wait that ran out) are written to the
+ *     caller's `dev_status` word (device, int32, OR-ed bit mask of 1 << moe_status; the
+ *     caller zeroes it) and the kernels return normally; outputs are then unspecified but
+ *     every access stays in bounds.
+ *   - Ties (the paper is silent): inside a token the lower expert id ranks first; inside the
+ *     Alloc-T pool the lower flat index t*K_orig + j ranks first.  With rows sorted
+ *     descending the kept pairs of token t are its columns 0 .. n_sel[t]-1.
+ */
+#ifndef ALLOCMOE_H_
+#define ALLOCMOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MOE_OK = 0,
+  MOE_ERR_ARG = 1,        /* null / misaligned pointer, unsupported shape */
+  MOE_ERR_BUDGET = 2,     /* budget outside [K_base*T, K_orig*T], or sum n_sel != budget */
+  MOE_ERR_WORKSPACE = 3,  /* workspace too small */
+  MOE_ERR_CUDA = 4,       /* a CUDA runtime / driver call failed */
+  MOE_ERR_NONFINITE = 5,  /* a routing score is NaN, Inf or negative */
+  MOE_ERR_TIMEOUT = 6     /* a bounded device-side wait gave up */
+} moe_status;
+
+/* T tokens, H hidden size, N routed experts, I expert intermediate size, S shared experts,
+ * K_orig nominal Top-K (candidates per token), K_base guaranteed experts per token (Eq. 10).
+ * Supported: H % 64 == 0, I % 64 == 0, 8 <= N <= 128 with N % 8 == 0, 1 <= K_orig <= min(N, 16),
+ * 0 <= K_base <= K_orig, S >= 0, T >= 1, T*K_orig < 2^31.  flags must be 0. */
+typedef struct {
+  int32_t T, H, N, I, S, K_orig, K_base;
+  uint32_t flags;
+} moe_shape;
+
+const char* moe_status_string(moe_status s);
+
+/* Bytes of device scratch that any call below needs for this shape with budgets up to
+ * budget_max (0 on an invalid shape). */
+size_t moe_workspace_bytes(const moe_shape* shape, int64_t budget_max);
+
+/* Eq. 1.  logits = x . W_gate (+ gate_bias), fp32 accumulation; scores = row softmax over all
+ * N experts in fp32; per token the K_orig largest scores, sorted descending (ties: lower expert
+ * id first).
+ *   x          device bf16 [T,H]
+ *   W_gate     device bf16 [H,N]      (the paper's W_gate in R^{H x N})
+ *   gate_bias  device fp32 [N] or NULL: added to the logits before the softmax
+ *   scores     device fp32 [T,N] or NULL (full softmax output, optional)
+ *   topk_idx   device int32 [T,K_orig]
+ *   topk_score device fp32 [T,K_orig] */
+moe_status moe_gate(const moe_shape* shape, const uint16_t* x, const uint16_t* W_gate,
+                    const float* gate_bias, float* scores, int32_t* topk_idx, float* topk_score,
+                    void* stream);
+
+/* Alloc-T (Sec. 3.3).  Input rows sorted descending; output n_sel[t] in [K_base, K_orig] with
+ * sum n_sel = budget: K_base plus the number of token t's residual scores among the
+ * budget - K_base*T largest of the pool.  Exact: scores are compared as values (their IEEE bit
+ * patterns, which order identically for non-negative floats), ties by flat index.
+ *   topk_score device fp32 [T,K_orig]
+ *   n_sel      device int32 [T]
+ *   dev_status device int32 [1]  (see above)
+ *   ws         device scratch, ws_bytes >= moe_workspace_bytes() */
+moe_status alloc_t_select(const moe_shape* shape, const float* topk_score, int64_t budget,
+                          int32_t* n_sel, int32_t* dev_status, void* ws, size_t ws_bytes,
+                          void* stream);
+
+/* Lists the kept pairs expert-ascending and token-ascending inside an expert.
+ *   expert_offsets device int32 [N+1]   exclusive prefix of per-expert counts, [N] = budget
+ *   perm_token     device int32 [budget] token of each listed pair
+ *   perm_weight    device fp32  [budget] its routing score
+ *   pair_pos       device int32 [T,K_orig] list position of pair (t,j), -1 if not kept
+ *   x_perm         device bf16 [budget,H] or NULL: row p is x[perm_token[p]] */
+moe_status moe_permute(const moe_shape* shape, const uint16_t* x, const int32_t* topk_idx,
+                       const float* topk_score, const int32_t* n_sel, int64_t budget,
+                       int32_t* expert_offsets, int32_t* perm_token, float* perm_weight,
+                       int32_t* pair_pos, uint16_t* x_perm, int32_t* dev_status,
+                       void* ws, size_t ws_bytes, void* stream);
+
+/* Routed experts ("each activated expert corresponds to one feed-forward execution",
+ * Sec. 3.1).  For every listed pair p of expert e:
+ *   h = silu(x_p W1_e^T) * (x_p W3_e^T)  (fp32 accumulation, h stored as bf16)
+ *   y_perm[p] = h W2_e^T                 (fp32 accumulation, stored as bf16)
+ *   x_perm  device bf16 [budget,H]  rows in list order (moe_permute's x_perm)
+ *   W13     device bf16 [N,2I,H]    rows 0..I-1 of an expert are W1, rows I..2I-1 are W3
+ *   W2      device bf16 [N,H,I]
+ *   y_perm  device bf16 [budget,H]
+ * Experts with no rows read no weights. */
+moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_perm,
+                           const int32_t* expert_offsets, int64_t budget, const uint16_t* W13,
+                           const uint16_t* W2, uint16_t* y_perm, int32_t* dev_status, void* ws,
+                           size_t ws_bytes, void* stream);
+
+/* Shared experts: y_shared[t] = sum_s E^sh_s(x_t) for every token (weight 1, outside the
+ * budget; a workload parameter, the paper's budgets count routed experts only).
+ *   Wsh13 device bf16 [S,2I,H], Wsh2 device bf16 [S,H,I], y_shared device bf16 [T,H] */
+moe_status moe_shared_ffn(const moe_shape* shape, const uint16_t* x, const uint16_t* Wsh13,
+                          const uint16_t* Wsh2, uint16_t* y_shared, int32_t* dev_status, void* ws,
+                          size_t ws_bytes, void* stream);
+
+/* Eq. 2 over the kept pairs: out[t] = sum_{j<n_sel[t]} topk_score[t,j] * y_perm[pair_pos[t,j]]
+ * (+ y_shared[t]); fp32, j ascending, one rounding to bf16.
+ *   y_shared device bf16 [T,H] or NULL;  out device bf16 [T,H] */
+moe_status moe_combine(const moe_shape* shape, const uint16_t* y_perm, const int32_t* pair_pos,
+                       const float* topk_score, const int32_t* n_sel, const uint16_t* y_shared,
+                       uint16_t* out, void* stream);
+
+/* The whole layer on one stream: moe_gate, alloc_t_select, moe_permute, moe_grouped_ffn
+ * (+ moe_shared_ffn when S > 0), moe_combine; all intermediates live in `ws`.
+ * Wsh13 / Wsh2 are ignored when S == 0.  With residual != 0 the layer input is added:
+ * out = x + MoE(x) (fp32 add, one bf16 rounding), the step of a residual layer stack. */
+moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const uint16_t* W_gate,
+                             const float* gate_bias, const uint16_t* W13, const uint16_t* W2,
+                             const uint16_t* Wsh13, const uint16_t* Wsh2, int64_t budget,
+                             int32_t residual, uint16_t* out, int32_t* dev_status, void* ws,
+                             size_t ws_bytes, void* stream);
+
+/* Device addresses of the routing intermediates that moe_layer_forward, called with this shape,
+ * this budget and this workspace, leaves in `ws` (for inspection and tests; valid until ws is
+ * reused; the carve-up depends on the budget).  Any output pointer may be NULL. */
+moe_status moe_layer_intermediates(const moe_shape* shape, int64_t budget, void* ws,
+                                   size_t ws_bytes, int32_t** topk_idx, float** topk_score,
+                                   int32_t** n_sel, int32_t** expert_offsets,
+                                   int32_t** perm_token, int32_t** pair_pos, uint16_t** y_perm);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ALLOCMOE_H_ */

@@ -1,0 +1,214 @@
+// C-ABI entry points (see include/allocmoe.h): argument checks, workspace carve-up, launches.
+// Nothing here allocates or synchronises; every launch goes to the caller's stream.
+#include <cuda_runtime.h>
+
+#include "allocmoe.h"
+
+// launchers defined next to their kernels
+moe_status launch_moe_gate(const moe_shape*, const uint16_t*, const uint16_t*, const float*, float*, int32_t*, float*,
+                           cudaStream_t);
+moe_status launch_alloc_t_select(const moe_shape*, const float*, int64_t, int32_t*, int32_t*, cudaStream_t);
+moe_status launch_moe_permute(const moe_shape*, const uint16_t*, const int32_t*, const float*, const int32_t*, int64_t,
+                              int32_t*, int32_t*, float*, int32_t*, uint16_t*, int32_t*, int32_t*, cudaStream_t);
+moe_status launch_ffn(const moe_shape*, const uint16_t*, const int32_t*, int64_t, const uint16_t*, const uint16_t*,
+                      uint16_t*, uint16_t*, const uint16_t*, const uint16_t*, const uint16_t*, uint16_t*, uint16_t*,
+                      int32_t*, cudaStream_t);
+moe_status launch_moe_combine(const moe_shape*, const uint16_t*, const int32_t*, const float*, const int32_t*,
+                              const uint16_t*, const uint16_t*, long long, uint16_t*, cudaStream_t);
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool shape_ok(const moe_shape* s) {
+  if (s == nullptr) return false;
+  if (s->flags != 0) return false;
+  if (s->T < 1 || s->H < 64 || s->I < 64 || s->N < 8 || s->S < 0) return false;
+  if (s->H % 64 != 0 || s->I % 64 != 0 || s->N % 8 != 0 || s->N > 128) return false;
+  if (s->K_orig < 1 || s->K_orig > 16 || s->K_orig > s->N) return false;
+  if (s->K_base < 0 || s->K_base > s->K_orig) return false;
+  if ((long long)s->T * s->K_orig >= (1ll << 31)) return false;
+  return true;
+}
+
+bool budget_ok(const moe_shape* s, int64_t budget) {
+  return budget >= (int64_t)s->K_base * s->T && budget <= (int64_t)s->K_orig * s->T;
+}
+
+// Fixed carve-up of the workspace; every region starts on a 256-byte boundary.
+struct WsLayout {
+  size_t topk_idx, topk_score, n_sel, expert_offsets, perm_token, perm_weight, pair_pos, seg_counts;
+  size_t x_perm, h, y_perm, h_sh, y_shared, total;
+};
+
+WsLayout ws_layout(const moe_shape* s, int64_t budget_max) {
+  WsLayout L{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t at = off;
+    off += (bytes + 255) & ~(size_t)255;
+    return at;
+  };
+  const size_t T = s->T, H = s->H, N = s->N, I = s->I, S = s->S, K = s->K_orig, B = (size_t)budget_max;
+  L.topk_idx = take(T * K * 4);
+  L.topk_score = take(T * K * 4);
+  L.n_sel = take(T * 4);
+  L.expert_offsets = take((N + 1) * 4);
+  L.perm_token = take(B * 4);
+  L.perm_weight = take(B * 4);
+  L.pair_pos = take(T * K * 4);
+  L.seg_counts = take(N * ((T + 31) / 32) * 4);
+  L.x_perm = take(B * H * 2);
+  L.h = take(B * I * 2);
+  L.y_perm = take(B * H * 2);
+  L.h_sh = take(T * S * I * 2);
+  L.y_shared = take(T * H * 2);
+  L.total = off;
+  return L;
+}
+
+template <typename T>
+T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<unsigned char*>(ws) + off); }
+
+}  // namespace
+
+extern "C" {
+
+const char* moe_status_string(moe_status s) {
+  switch (s) {
+    case MOE_OK: return "ok";
+    case MOE_ERR_ARG: return "invalid argument (null or misaligned pointer, unsupported shape)";
+    case MOE_ERR_BUDGET: return "budget outside [K_base*T, K_orig*T] or kept counts do not add up to it";
+    case MOE_ERR_WORKSPACE: return "workspace too small";
+    case MOE_ERR_CUDA: return "CUDA call failed";
+    case MOE_ERR_NONFINITE: return "routing score is NaN, Inf or negative";
+    case MOE_ERR_TIMEOUT: return "bounded device wait gave up";
+  }
+  return "unknown status";
+}
+
+size_t moe_workspace_bytes(const moe_shape* shape, int64_t budget_max) {
+  if (!shape_ok(shape) || budget_max < 0 || budget_max > (int64_t)shape->K_orig * shape->T) return 0;
+  return ws_layout(shape, budget_max).total;
+}
+
+moe_status moe_gate(const moe_shape* shape, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,
+                    float* scores, int32_t* topk_idx, float* topk_score, void* stream) {
+  if (!shape_ok(shape) || !x || !W_gate || !topk_idx || !topk_score) return MOE_ERR_ARG;
+  if (!aligned16(x) || !aligned16(W_gate) || !aligned16(topk_idx) || !aligned16(topk_score)) return MOE_ERR_ARG;
+  return launch_moe_gate(shape, x, W_gate, gate_bias, scores, topk_idx, topk_score, (cudaStream_t)stream);
+}
+
+moe_status alloc_t_select(const moe_shape* shape, const float* topk_score, int64_t budget, int32_t* n_sel,
+                          int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  (void)ws;
+  (void)ws_bytes;
+  if (!shape_ok(shape) || !topk_score || !n_sel || !dev_status) return MOE_ERR_ARG;
+  if (!aligned16(topk_score) || !aligned16(n_sel)) return MOE_ERR_ARG;
+  if (!budget_ok(shape, budget)) return MOE_ERR_BUDGET;
+  return launch_alloc_t_select(shape, topk_score, budget, n_sel, dev_status, (cudaStream_t)stream);
+}
+
+moe_status moe_permute(const moe_shape* shape, const uint16_t* x, const int32_t* topk_idx, const float* topk_score,
+                       const int32_t* n_sel, int64_t budget, int32_t* expert_offsets, int32_t* perm_token,
+                       float* perm_weight, int32_t* pair_pos, uint16_t* x_perm, int32_t* dev_status, void* ws,
+                       size_t ws_bytes, void* stream) {
+  if (!shape_ok(shape) || !topk_idx || !topk_score || !n_sel || !expert_offsets || !perm_token || !perm_weight ||
+      !pair_pos || !dev_status || !ws)
+    return MOE_ERR_ARG;
+  if (x_perm != nullptr && (!x || !aligned16(x) || !aligned16(x_perm))) return MOE_ERR_ARG;
+  if (!aligned16(ws)) return MOE_ERR_ARG;
+  if (!budget_ok(shape, budget)) return MOE_ERR_BUDGET;
+  const WsLayout L = ws_layout(shape, budget);
+  if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
+  return launch_moe_permute(shape, x, topk_idx, topk_score, n_sel, budget, expert_offsets, perm_token, perm_weight,
+                            pair_pos, x_perm, dev_status, at<int32_t>(ws, L.seg_counts), (cudaStream_t)stream);
+}
+
+moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_perm, const int32_t* expert_offsets,
+                           int64_t budget, const uint16_t* W13, const uint16_t* W2, uint16_t* y_perm,
+                           int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  if (!shape_ok(shape) || !x_perm || !expert_offsets || !W13 || !W2 || !y_perm || !dev_status || !ws) return MOE_ERR_ARG;
+  if (!aligned16(x_perm) || !aligned16(W13) || !aligned16(W2) || !aligned16(y_perm) || !aligned16(ws)) return MOE_ERR_ARG;
+  if (budget < 0 || budget > (int64_t)shape->K_orig * shape->T) return MOE_ERR_BUDGET;
+  const WsLayout L = ws_layout(shape, budget);
+  if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
+  return launch_ffn(shape, x_perm, expert_offsets, budget, W13, W2, at<uint16_t>(ws, L.h), y_perm, nullptr, nullptr,
+                    nullptr, nullptr, nullptr, dev_status, (cudaStream_t)stream);
+}
+
+moe_status moe_shared_ffn(const moe_shape* shape, const uint16_t* x, const uint16_t* Wsh13, const uint16_t* Wsh2,
+                          uint16_t* y_shared, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  if (!shape_ok(shape) || shape->S < 1 || !x || !Wsh13 || !Wsh2 || !y_shared || !dev_status || !ws) return MOE_ERR_ARG;
+  if (!aligned16(x) || !aligned16(Wsh13) || !aligned16(Wsh2) || !aligned16(y_shared) || !aligned16(ws)) return MOE_ERR_ARG;
+  const WsLayout L = ws_layout(shape, 0);
+  if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
+  return launch_ffn(shape, nullptr, nullptr, 0, nullptr, nullptr, nullptr, nullptr, x, Wsh13, Wsh2,
+                    at<uint16_t>(ws, L.h_sh), y_shared, dev_status, (cudaStream_t)stream);
+}
+
+moe_status moe_combine(const moe_shape* shape, const uint16_t* y_perm, const int32_t* pair_pos,
+                       const float* topk_score, const int32_t* n_sel, const uint16_t* y_shared, uint16_t* out,
+                       void* stream) {
+  if (!shape_ok(shape) || !y_perm || !pair_pos || !topk_score || !n_sel || !out) return MOE_ERR_ARG;
+  if (!aligned16(y_perm) || !aligned16(out) || (y_shared && !aligned16(y_shared))) return MOE_ERR_ARG;
+  return launch_moe_combine(shape, y_perm, pair_pos, topk_score, n_sel, y_shared, nullptr,
+                            (long long)shape->K_orig * shape->T, out, (cudaStream_t)stream);
+}
+
+moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,
+                             const uint16_t* W13, const uint16_t* W2, const uint16_t* Wsh13, const uint16_t* Wsh2,
+                             int64_t budget, int32_t residual, uint16_t* out, int32_t* dev_status, void* ws,
+                             size_t ws_bytes, void* stream) {
+  if (!shape_ok(shape) || !x || !W_gate || !W13 || !W2 || !out || !dev_status || !ws) return MOE_ERR_ARG;
+  if (shape->S > 0 && (!Wsh13 || !Wsh2)) return MOE_ERR_ARG;
+  if (!aligned16(x) || !aligned16(W_gate) || !aligned16(W13) || !aligned16(W2) || !aligned16(out) || !aligned16(ws))
+    return MOE_ERR_ARG;
+  if (shape->S > 0 && (!aligned16(Wsh13) || !aligned16(Wsh2))) return MOE_ERR_ARG;
+  if (!budget_ok(shape, budget)) return MOE_ERR_BUDGET;
+  const WsLayout L = ws_layout(shape, budget);
+  if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  int32_t* topk_idx = at<int32_t>(ws, L.topk_idx);
+  float* topk_score = at<float>(ws, L.topk_score);
+  int32_t* n_sel = at<int32_t>(ws, L.n_sel);
+  int32_t* expert_offsets = at<int32_t>(ws, L.expert_offsets);
+  int32_t* perm_token = at<int32_t>(ws, L.perm_token);
+  float* perm_weight = at<float>(ws, L.perm_weight);
+  int32_t* pair_pos = at<int32_t>(ws, L.pair_pos);
+  uint16_t* x_perm = at<uint16_t>(ws, L.x_perm);
+  uint16_t* y_perm = at<uint16_t>(ws, L.y_perm);
+  uint16_t* y_shared = shape->S > 0 ? at<uint16_t>(ws, L.y_shared) : nullptr;
+
+  moe_status r = launch_moe_gate(shape, x, W_gate, gate_bias, nullptr, topk_idx, topk_score, st);
+  if (r != MOE_OK) return r;
+  r = launch_alloc_t_select(shape, topk_score, budget, n_sel, dev_status, st);
+  if (r != MOE_OK) return r;
+  r = launch_moe_permute(shape, x, topk_idx, topk_score, n_sel, budget, expert_offsets, perm_token, perm_weight,
+                         pair_pos, x_perm, dev_status, at<int32_t>(ws, L.seg_counts), st);
+  if (r != MOE_OK) return r;
+  r = launch_ffn(shape, x_perm, expert_offsets, budget, W13, W2, at<uint16_t>(ws, L.h), y_perm,
+                 shape->S > 0 ? x : nullptr, Wsh13, Wsh2, at<uint16_t>(ws, L.h_sh), y_shared, dev_status, st);
+  if (r != MOE_OK) return r;
+  return launch_moe_combine(shape, y_perm, pair_pos, topk_score, n_sel, y_shared, residual ? x : nullptr, budget, out,
+                            st);
+}
+
+moe_status moe_layer_intermediates(const moe_shape* shape, int64_t budget_max, void* ws, size_t ws_bytes,
+                                   int32_t** topk_idx, float** topk_score, int32_t** n_sel, int32_t** expert_offsets,
+                                   int32_t** perm_token, int32_t** pair_pos, uint16_t** y_perm) {
+  if (!shape_ok(shape) || !ws) return MOE_ERR_ARG;
+  if (budget_max < 0 || budget_max > (int64_t)shape->K_orig * shape->T) return MOE_ERR_BUDGET;
+  const WsLayout L = ws_layout(shape, budget_max);
+  if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
+  if (topk_idx) *topk_idx = at<int32_t>(ws, L.topk_idx);
+  if (topk_score) *topk_score = at<float>(ws, L.topk_score);
+  if (n_sel) *n_sel = at<int32_t>(ws, L.n_sel);
+  if (expert_offsets) *expert_offsets = at<int32_t>(ws, L.expert_offsets);
+  if (perm_token) *perm_token = at<int32_t>(ws, L.perm_token);
+  if (pair_pos) *pair_pos = at<int32_t>(ws, L.pair_pos);
+  if (y_perm) *y_perm = at<uint16_t>(ws, L.y_perm);
+  return MOE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,72 @@
+// moe_combine: Eq. 2 over the kept pairs.
+//   out[t] = sum_{j < n_sel[t]} topk_score[t,j] * y_perm[pair_pos[t,j]]  (+ y_shared[t]) (+ x[t])
+// fp32 FMAs in ascending j, one rounding to bf16.  One CTA per token, 16 bytes (8 bf16) per
+// thread per step: every global access is a coalesced 128-bit load or store.
+#include "common.cuh"
+
+namespace allocmoe {
+
+DEV void fma8(float (&acc)[8], const uint4& v, float w) {
+  const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    acc[2 * q] = fmaf(w, bf16_bits_to_float(u[q] & 0xFFFFu), acc[2 * q]);
+    acc[2 * q + 1] = fmaf(w, bf16_bits_to_float(u[q] >> 16), acc[2 * q + 1]);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+combine_kernel(const uint4* __restrict__ y_perm, const int32_t* __restrict__ pair_pos,
+               const float* __restrict__ topk_score, const int32_t* __restrict__ n_sel,
+               const uint4* __restrict__ y_shared, const uint4* __restrict__ x_res, int K_orig, int row_vec,
+               long long budget_rows, uint4* __restrict__ out) {
+  __shared__ int s_pos[16];
+  __shared__ float s_w[16];
+  __shared__ int s_n;
+  const int t = blockIdx.x;
+  if (threadIdx.x < 16) {
+    const int j = threadIdx.x;
+    const int n = min(max(n_sel[t], 0), K_orig);
+    if (j == 0) s_n = n;
+    int pos = -1;
+    float w = 0.f;
+    if (j < n) {
+      pos = pair_pos[(long long)t * K_orig + j];
+      w = topk_score[(long long)t * K_orig + j];
+      if (pos < 0 || pos >= budget_rows) { pos = -1; w = 0.f; }
+    }
+    s_pos[j] = pos;
+    s_w[j] = w;
+  }
+  __syncthreads();
+  const int n = s_n;
+  for (int c = threadIdx.x; c < row_vec; c += blockDim.x) {
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int j = 0; j < n; ++j) {
+      const int pos = s_pos[j];
+      if (pos >= 0) fma8(acc, __ldg(y_perm + (long long)pos * row_vec + c), s_w[j]);
+    }
+    if (y_shared != nullptr) fma8(acc, __ldg(y_shared + (long long)t * row_vec + c), 1.f);
+    if (x_res != nullptr) fma8(acc, __ldg(x_res + (long long)t * row_vec + c), 1.f);
+    uint4 o;
+    o.x = pack_bf16x2(acc[0], acc[1]);
+    o.y = pack_bf16x2(acc[2], acc[3]);
+    o.z = pack_bf16x2(acc[4], acc[5]);
+    o.w = pack_bf16x2(acc[6], acc[7]);
+    out[(long long)t * row_vec + c] = o;
+  }
+}
+
+}  // namespace allocmoe
+
+using namespace allocmoe;
+
+moe_status launch_moe_combine(const moe_shape* s, const uint16_t* y_perm, const int32_t* pair_pos,
+                              const float* topk_score, const int32_t* n_sel, const uint16_t* y_shared,
+                              const uint16_t* x_res, long long budget_rows, uint16_t* out, cudaStream_t stream) {
+  combine_kernel<<<s->T, 256, 0, stream>>>(reinterpret_cast<const uint4*>(y_perm), pair_pos, topk_score, n_sel,
+                                           reinterpret_cast<const uint4*>(y_shared),
+                                           reinterpret_cast<const uint4*>(x_res), s->K_orig, s->H / 8, budget_rows,
+                                           reinterpret_cast<uint4*>(out));
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}

@@ -1,0 +1,430 @@
+// Grouped SwiGLU expert GEMMs on the 5th-generation tensor cores (tcgen05 + TMEM), fed by TMA.
+//
+// "Each activated expert corresponds to one feed-forward execution" (Sec. 3.1): for the rows of
+// expert e (a contiguous run of the permuted list)
+//     GEMM-1   h = silu(X W1_e^T) * (X W3_e^T)       [rows, I]   (SwiGLU fused in the epilogue)
+//     GEMM-2   y = h W2_e^T                          [rows, H]
+// Both are C = A B^T with A [rows, K] and B [n, K] K-contiguous, i.e. both operands K-major.
+//
+// One persistent kernel per GEMM: grid = number of SMs, every CTA walks the tile list
+// tile = blockIdx.x, += gridDim.x.  The list is built on the device from expert_offsets (row
+// counts are data dependent): groups in order, inside a group column blocks outermost and
+// 128-row blocks innermost, so CTAs that run concurrently share a weight tile through L2.
+// A "group" is a routed expert or, last, the shared experts (all T rows; their S sub-experts
+// are extra column blocks in GEMM-1 and extra K blocks in GEMM-2).
+//
+// CTA = 6 warps: warp 0 lane 0 issues TMA loads (A 128x64, B 256x64 bf16, 128-byte swizzle)
+// into a 4-stage ring; warp 1 lane 0 issues tcgen05.mma (M=128, N=256, K=16) into one of two
+// 256-column TMEM accumulators; warps 2-5 read the finished accumulator with tcgen05.ld, apply
+// the epilogue and store bf16 rows (row-masked at the ragged end of an expert's run) while the
+// next tile's main loop runs.  Every mbarrier wait is bounded (see common.cuh).
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace allocmoe {
+
+constexpr int kBM = 128;            // rows per tile (UMMA M)
+constexpr int kBK = 64;             // K per stage: 64 bf16 = one 128-byte swizzle row
+constexpr int kUmmaN = 256;         // accumulator columns per tile
+constexpr int kStages = 4;
+constexpr int kFfnThreads = 192;
+constexpr int kABytes = kBM * kBK * 2;        // 16 KB
+constexpr int kBBytes = kUmmaN * kBK * 2;     // 32 KB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kTmemCols = 512;      // two accumulators of 256 columns
+constexpr int kMaxGroups = 130;     // up to 128 routed experts + the shared group
+
+struct FfnGemmParams {
+  const int32_t* expert_offsets;    // device [n_experts+1]; unused when n_experts == 0
+  int n_experts;                    // routed groups
+  int shared_rows;                  // T when the shared group is present, else 0
+  int shared_sub;                   // S
+  int n_per_sub;                    // output columns per (sub-)expert: I for GEMM-1, H for GEMM-2
+  int k_per_sub;                    // K per (sub-)expert: H for GEMM-1, I for GEMM-2
+  int up_row_offset;                // GEMM-1: row of W3 inside an expert's W13 (= I)
+  __nv_bfloat16* out_routed;        // GEMM-1: h [rows, I]; GEMM-2: y_perm [rows, H]
+  __nv_bfloat16* out_shared;        // GEMM-1: h_sh [T, S*I]; GEMM-2: y_shared [T, H]
+  long long ld_out_routed, ld_out_shared;
+  int32_t* dev_status;
+};
+
+struct FfnSmemCtl {
+  uint64_t full[kStages];
+  uint64_t empty[kStages];
+  uint64_t tmem_full[2];
+  uint64_t tmem_empty[2];
+  uint64_t drain;
+  uint32_t tmem_base;
+  volatile int abort_flag;
+  int n_groups;
+  int total_tiles;
+  int tile_start[kMaxGroups + 1];   // first tile of each group
+  int row_start[kMaxGroups];        // first row of each group in its A / output matrix
+  int row_count[kMaxGroups];
+};
+
+struct TileCoord {
+  int group, m0, m_end, nb;
+  bool shared;
+};
+
+// kSwiGLU: true = GEMM-1 (B tile = 128 W1 rows + 128 W3 rows, 128 output columns),
+//          false = GEMM-2 (B tile = 256 W2 rows, 256 output columns).
+template <bool kSwiGLU>
+struct TileWalker {
+  const FfnSmemCtl* c;
+  int nb_routed, nb_shared;
+  int g;
+  DEV TileWalker(const FfnSmemCtl* ctl, const FfnGemmParams& p) : c(ctl), g(0) {
+    constexpr int cols = kSwiGLU ? kUmmaN / 2 : kUmmaN;
+    nb_routed = (p.n_per_sub + cols - 1) / cols;
+    nb_shared = kSwiGLU ? nb_routed * p.shared_sub : nb_routed;
+  }
+  DEV TileCoord at(int tile, const FfnGemmParams& p) {
+    while (tile >= c->tile_start[g + 1]) ++g;   // tile < total_tiles, tile_start is non-decreasing
+    TileCoord tc;
+    tc.group = g;
+    tc.shared = (g >= p.n_experts);
+    const int local = tile - c->tile_start[g];
+    const int mblocks = (c->row_count[g] + kBM - 1) / kBM;
+    tc.nb = local / mblocks;
+    const int mb = local % mblocks;
+    tc.m0 = c->row_start[g] + mb * kBM;
+    tc.m_end = c->row_start[g] + c->row_count[g];
+    return tc;
+  }
+};
+
+template <bool kSwiGLU>
+__global__ void __launch_bounds__(kFfnThreads, 1)
+ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_routed,
+                const __grid_constant__ CUtensorMap tmB_routed, const __grid_constant__ CUtensorMap tmA_shared,
+                const __grid_constant__ CUtensorMap tmB_shared) {
+  extern __shared__ unsigned char smem_dyn[];
+  // tiles need 1024-byte alignment for the 128-byte swizzle
+  unsigned char* tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  FfnSmemCtl* ctl = reinterpret_cast<FfnSmemCtl*>(tiles + kStages * kStageBytes);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int kOutCols = kSwiGLU ? kUmmaN / 2 : kUmmaN;
+
+  // ---------------- setup: group table, barriers, TMEM
+  const int n_groups = p.n_experts + (p.shared_rows > 0 ? 1 : 0);
+  for (int gi = tid; gi < n_groups; gi += kFfnThreads) {
+    if (gi < p.n_experts) {
+      const int lo = p.expert_offsets[gi], hi = p.expert_offsets[gi + 1];
+      ctl->row_start[gi] = lo;
+      ctl->row_count[gi] = max(hi - lo, 0);
+    } else {
+      ctl->row_start[gi] = 0;
+      ctl->row_count[gi] = p.shared_rows;
+    }
+  }
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tmem_full[a], 1); mbar_init(&ctl->tmem_empty[a], 4); }
+    mbar_init(&ctl->drain, 1);
+    ctl->abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tensormap(&tmA_routed);
+    prefetch_tensormap(&tmB_routed);
+    prefetch_tensormap(&tmA_shared);
+    prefetch_tensormap(&tmB_shared);
+  }
+  __syncthreads();
+  if (tid == 0) {
+    TileWalker<kSwiGLU> w(ctl, p);
+    int acc = 0;
+    for (int gi = 0; gi < n_groups; ++gi) {
+      ctl->tile_start[gi] = acc;
+      const int mblocks = (ctl->row_count[gi] + kBM - 1) / kBM;
+      acc += mblocks * (gi < p.n_experts ? w.nb_routed : w.nb_shared);
+    }
+    ctl->tile_start[n_groups] = acc;
+    ctl->total_tiles = acc;
+    ctl->n_groups = n_groups;
+  }
+  if (warp == 1) {
+    tmem_alloc(&ctl->tmem_base, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = ctl->tmem_base;
+  const int total_tiles = ctl->total_tiles;
+  const int kb_routed = p.k_per_sub / kBK;
+  const int kb_shared = kSwiGLU ? kb_routed : kb_routed * p.shared_sub;
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  if (warp == 0) {
+    // ======================= TMA producer =======================
+    if (lane == 0) {
+      TileWalker<kSwiGLU> w(ctl, p);
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const TileCoord tc = w.at(tile, p);
+        const CUtensorMap* tmA = tc.shared ? &tmA_shared : &tmA_routed;
+        const CUtensorMap* tmB = tc.shared ? &tmB_shared : &tmB_routed;
+        const int nkb = tc.shared ? kb_shared : kb_routed;
+        // expert coordinate and row inside the expert's weight matrix for this column block
+        int e_n = tc.group, n_row = tc.nb * kOutCols;
+        if (tc.shared) {
+          if (kSwiGLU) { e_n = tc.nb / w.nb_routed; n_row = (tc.nb % w.nb_routed) * kOutCols; }
+          else { e_n = 0; }
+        }
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!(ok = mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status))) break;
+          unsigned char* sa = tiles + s * kStageBytes;
+          unsigned char* sb = sa + kABytes;
+          mbar_expect_tx(&ctl->full[s], kStageBytes);
+          tma_load_2d(sa, tmA, &ctl->full[s], kb * kBK, tc.m0);
+          int e_k = e_n, k_col = kb * kBK;
+          if (tc.shared && !kSwiGLU) { e_k = kb / kb_routed; k_col = (kb % kb_routed) * kBK; }
+          if (kSwiGLU) {
+            tma_load_3d(sb, tmB, &ctl->full[s], k_col, n_row, e_k);
+            tma_load_3d(sb + kBBytes / 2, tmB, &ctl->full[s], k_col, p.up_row_offset + n_row, e_k);
+          } else {
+            tma_load_3d(sb, tmB, &ctl->full[s], k_col, n_row, e_k);
+          }
+        }
+      }
+      // drain: every load this thread issued must have landed before the CTA may exit
+      const uint32_t issued = it;
+      for (uint32_t q = (issued > (uint32_t)kStages ? issued - kStages : 0u); q < issued; ++q)
+        mbar_wait_drain(&ctl->full[q % kStages], (q / kStages) & 1u);
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ======================= MMA issuer =======================
+    if (lane == 0) {
+      TileWalker<kSwiGLU> w(ctl, p);
+      constexpr uint32_t idesc = umma_idesc_bf16(kBM, kUmmaN);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+        const TileCoord tc = w.at(tile, p);
+        const int nkb = tc.shared ? kb_shared : kb_routed;
+        const uint32_t a = tcount & 1u, aph = (tcount >> 1) & 1u;
+        if (!(ok = mbar_wait_bounded(&ctl->tmem_empty[a], aph ^ 1u, abort_flag, p.dev_status))) break;
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + a * kUmmaN;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!(ok = mbar_wait_bounded(&ctl->full[s], ph, abort_flag, p.dev_status))) break;
+          tc_fence_after_sync();
+          const uint32_t sa = smem_u32(tiles + s * kStageBytes);
+          const uint64_t da = umma_desc_sw128(sa), db = umma_desc_sw128(sa + kABytes);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k)
+            umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+          umma_commit(&ctl->empty[s]);      // frees the stage once these MMAs have read it
+        }
+        if (ok) umma_commit(&ctl->tmem_full[a]);
+      }
+      // drain: all MMAs complete before TMEM is freed
+      umma_commit(&ctl->drain);
+      mbar_wait_drain(&ctl->drain, 0u);
+    }
+    __syncwarp();
+  } else {
+    // ======================= epilogue (warps 2..5) =======================
+    TileWalker<kSwiGLU> w(ctl, p);
+    const int q = warp & 3;                  // TMEM lane quarter this warp may read
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+      const TileCoord tc = w.at(tile, p);
+      const uint32_t a = tcount & 1u, aph = (tcount >> 1) & 1u;
+      if (!(ok = mbar_wait_bounded(&ctl->tmem_full[a], aph, abort_flag, p.dev_status))) break;
+      tc_fence_after_sync();
+      const int row = tc.m0 + q * 32 + lane;
+      const bool row_ok = row < tc.m_end;
+      const int n_total = tc.shared ? (kSwiGLU ? p.n_per_sub * p.shared_sub : p.n_per_sub) : p.n_per_sub;
+      int col0 = tc.nb * kOutCols;           // first output column of the tile
+      int col_limit = n_total;
+      if (kSwiGLU && tc.shared) {            // column block nb of sub-expert s -> column s*I + ...
+        const int s = tc.nb / w.nb_routed;
+        col0 = s * p.n_per_sub + (tc.nb % w.nb_routed) * kOutCols;
+        col_limit = (s + 1) * p.n_per_sub;
+      }
+      __nv_bfloat16* out = tc.shared ? p.out_shared : p.out_routed;
+      const long long ld = tc.shared ? p.ld_out_shared : p.ld_out_routed;
+      __nv_bfloat16* out_row = out + (long long)row * ld;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * kUmmaN;
+#pragma unroll 1
+      for (int c = 0; c < kOutCols / 32; ++c) {
+        uint32_t packed[16];
+        if (kSwiGLU) {
+          uint32_t g[32], u[32];
+          tmem_ld_32x32(taddr + c * 32, g);
+          tmem_ld_32x32(taddr + kUmmaN / 2 + c * 32, u);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+            const float h0 = g0 * __uint_as_float(u[2 * i]) / (1.f + __expf(-g0));
+            const float h1 = g1 * __uint_as_float(u[2 * i + 1]) / (1.f + __expf(-g1));
+            packed[i] = pack_bf16x2(h0, h1);
+          }
+        } else {
+          uint32_t v[32];
+          tmem_ld_32x32(taddr + c * 32, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) packed[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+        }
+        const int col = col0 + c * 32;
+        if (row_ok) {
+          if (col + 32 <= col_limit) {
+            uint4* dst = reinterpret_cast<uint4*>(out_row + col);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+          } else {
+            for (int i = 0; i < 32; ++i)
+              if (col + i < col_limit) {
+                const uint32_t w2 = packed[i >> 1];
+                reinterpret_cast<uint16_t*>(out_row)[col + i] = (uint16_t)((i & 1) ? (w2 >> 16) : (w2 & 0xFFFFu));
+              }
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ctl->tmem_empty[a]);
+    }
+  }
+
+  // ---------------- teardown
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace allocmoe
+
+using namespace allocmoe;
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 tensor [d2][d1][d0] (d0 contiguous), box {64, box1, 1}, 128-byte swizzle, zero fill.
+static bool make_tmap(CUtensorMap* tm, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1_elems,
+                      uint64_t stride2_elems, uint32_t box1) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[3] = {d0, d1, d2};
+  cuuint64_t strides[2] = {stride1_elems * 2, stride2_elems * 2};
+  cuuint32_t box[3] = {(cuuint32_t)kBK, box1, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  const int rank = d2 > 0 ? 3 : 2;
+  if (rank == 2) dims[2] = 1;
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int g_num_sms = 0;
+static int num_sms() {
+  if (g_num_sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (g_num_sms <= 0) g_num_sms = 148;
+  }
+  return g_num_sms;
+}
+
+constexpr size_t kFfnSmemBytes = (size_t)kStages * kStageBytes + sizeof(FfnSmemCtl) + 1024;
+
+template <bool kSwiGLU>
+static moe_status launch_gemm(const FfnGemmParams& p, const CUtensorMap& ar, const CUtensorMap& br,
+                              const CUtensorMap& as, const CUtensorMap& bs, cudaStream_t stream) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(ffn_gemm_kernel<kSwiGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kFfnSmemBytes) != cudaSuccess)
+      return MOE_ERR_CUDA;
+    attr_done = true;
+  }
+  ffn_gemm_kernel<kSwiGLU><<<num_sms(), kFfnThreads, kFfnSmemBytes, stream>>>(p, ar, br, as, bs);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+// Routed and/or shared experts in one pair of launches.
+//   routed part present iff budget > 0 && x_perm != nullptr; shared part iff S > 0 && x_shared != nullptr.
+moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t* expert_offsets, int64_t budget,
+                      const uint16_t* W13, const uint16_t* W2, uint16_t* h, uint16_t* y_perm, const uint16_t* x_shared,
+                      const uint16_t* Wsh13, const uint16_t* Wsh2, uint16_t* h_sh, uint16_t* y_shared,
+                      int32_t* dev_status, cudaStream_t stream) {
+  const bool routed = (budget > 0 && x_perm != nullptr);
+  const bool shared = (s->S > 0 && x_shared != nullptr);
+  if (!routed && !shared) return MOE_OK;
+  const uint64_t H = s->H, I = s->I;
+  CUtensorMap a1r, b1r, a1s, b1s, a2r, b2r, a2s, b2s;
+  bool ok = true;
+  if (routed) {
+    ok &= make_tmap(&a1r, x_perm, H, (uint64_t)budget, 0, H, 0, kBM);
+    ok &= make_tmap(&b1r, W13, H, 2 * I, (uint64_t)s->N, H, 2 * I * H, kUmmaN / 2);
+    ok &= make_tmap(&a2r, h, I, (uint64_t)budget, 0, I, 0, kBM);
+    ok &= make_tmap(&b2r, W2, I, H, (uint64_t)s->N, I, H * I, kUmmaN);
+  }
+  if (shared) {
+    const uint64_t S = s->S;
+    ok &= make_tmap(&a1s, x_shared, H, (uint64_t)s->T, 0, H, 0, kBM);
+    ok &= make_tmap(&b1s, Wsh13, H, 2 * I, S, H, 2 * I * H, kUmmaN / 2);
+    ok &= make_tmap(&a2s, h_sh, S * I, (uint64_t)s->T, 0, S * I, 0, kBM);
+    ok &= make_tmap(&b2s, Wsh2, I, H, S, I, H * I, kUmmaN);
+  }
+  if (!ok) return MOE_ERR_CUDA;
+  if (!routed) { a1r = a1s; b1r = b1s; a2r = a2s; b2r = b2s; }
+  if (!shared) { a1s = a1r; b1s = b1r; a2s = a2r; b2s = b2r; }
+
+  FfnGemmParams p{};
+  p.expert_offsets = expert_offsets;
+  p.n_experts = routed ? s->N : 0;
+  p.shared_rows = shared ? s->T : 0;
+  p.shared_sub = s->S;
+  p.dev_status = dev_status;
+  // GEMM-1
+  p.n_per_sub = s->I;
+  p.k_per_sub = s->H;
+  p.up_row_offset = s->I;
+  p.out_routed = reinterpret_cast<__nv_bfloat16*>(h);
+  p.out_shared = reinterpret_cast<__nv_bfloat16*>(h_sh);
+  p.ld_out_routed = s->I;
+  p.ld_out_shared = (long long)s->S * s->I;
+  moe_status st = launch_gemm<true>(p, a1r, b1r, a1s, b1s, stream);
+  if (st != MOE_OK) return st;
+  // GEMM-2
+  p.n_per_sub = s->H;
+  p.k_per_sub = s->I;
+  p.up_row_offset = 0;
+  p.out_routed = reinterpret_cast<__nv_bfloat16*>(y_perm);
+  p.out_shared = reinterpret_cast<__nv_bfloat16*>(y_shared);
+  p.ld_out_routed = s->H;
+  p.ld_out_shared = s->H;
+  return launch_gemm<false>(p, a2r, b2r, a2s, b2s, stream);
+}

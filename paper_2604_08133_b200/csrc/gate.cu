@@ -1,0 +1,244 @@
+// moe_gate: Eq. 1 fused -- logits = x . W_gate (+ bias), row softmax over all N experts (fp32),
+// and the K_orig largest scores per token sorted descending (ties: lower expert id first).
+//
+// The contraction is small (2*T*H*N flops; 1 GFLOP at T=4096, H=2048, N=64) and x is read once,
+// so the kernel is bound by streaming x from HBM and by latency.  A CTA owns 32 tokens and all N
+// experts; x and W_gate chunks of 128 along H are staged in shared memory with 16-byte cp.async
+// (3 stages) and multiplied with mma.sync m16n8k16 bf16 -> fp32 (the four warps split every
+// chunk's k-steps, their partial sums are added in a fixed order).  W_gate is stored [H,N]
+// (N contiguous, the paper's R^{H x N}), which is the "column" operand of mma.sync when read
+// with ldmatrix.trans.
+#include "common.cuh"
+
+namespace allocmoe {
+
+constexpr int kGateTM = 32;        // tokens per CTA
+constexpr int kGateKC = 128;       // H chunk
+constexpr int kGateStages = 3;
+constexpr int kGateThreads = 128;
+constexpr int kGateXStride = kGateKC + 8;   // bf16 elements per staged x row (272 B: conflict-free ldmatrix)
+
+DEV void ldmatrix_x4(uint32_t (&r)[4], const void* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(p)));
+}
+DEV void ldmatrix_x4_trans(uint32_t (&r)[4], const void* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(p)));
+}
+DEV void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// NT16 = number of 16-wide expert tiles (N padded to 16*NT16).
+template <int NT16>
+__global__ void __launch_bounds__(kGateThreads)
+moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ W_gate,
+                const float* __restrict__ gate_bias, int T, int H, int N, int K_orig, int w_stride,
+                float* __restrict__ scores, int32_t* __restrict__ topk_idx, float* __restrict__ topk_score) {
+  constexpr int NP = NT16 * 16;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int x_stage_bytes = kGateTM * kGateXStride * 2;
+  const int w_stage_bytes = kGateKC * w_stride * 2;
+  const int stage_bytes = x_stage_bytes + w_stage_bytes;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int t0 = blockIdx.x * kGateTM;
+  const int nchunks = (H + kGateKC - 1) / kGateKC;
+  const int n_vec = N / 8;   // 16-byte pieces per W_gate row
+
+  auto issue = [&](int chunk) {
+    if (chunk < nchunks) {
+      unsigned char* st = smem_raw + (chunk % kGateStages) * stage_bytes;
+      __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(st);
+      __nv_bfloat16* ws = reinterpret_cast<__nv_bfloat16*>(st + x_stage_bytes);
+      const int k0 = chunk * kGateKC;
+      for (int i = tid; i < kGateTM * (kGateKC / 8); i += kGateThreads) {
+        const int r = i / (kGateKC / 8), c = i % (kGateKC / 8);
+        const int t = t0 + r, k = k0 + c * 8;
+        const bool ok = (t < T) && (k < H);
+        cp_async_16(xs + r * kGateXStride + c * 8, x + (ok ? ((long long)t * H + k) : 0), ok);
+      }
+      for (int i = tid; i < kGateKC * (NP / 8); i += kGateThreads) {
+        const int r = i / (NP / 8), c = i % (NP / 8);
+        const int k = k0 + r;
+        const bool ok = (k < H) && (c < n_vec);
+        cp_async_16(ws + r * w_stride + c * 8, W_gate + (ok ? ((long long)k * N + c * 8) : 0), ok);
+      }
+    }
+    cp_async_commit();
+  };
+
+  float acc[2][NT16 * 2][4];
+#pragma unroll
+  for (int m = 0; m < 2; ++m)
+#pragma unroll
+    for (int n = 0; n < NT16 * 2; ++n)
+#pragma unroll
+      for (int q = 0; q < 4; ++q) acc[m][n][q] = 0.f;
+
+  issue(0);
+  issue(1);
+  for (int chunk = 0; chunk < nchunks; ++chunk) {
+    issue(chunk + 2);
+    cp_async_wait<2>();
+    __syncthreads();
+    const unsigned char* st = smem_raw + (chunk % kGateStages) * stage_bytes;
+    const __nv_bfloat16* xs = reinterpret_cast<const __nv_bfloat16*>(st);
+    const __nv_bfloat16* ws = reinterpret_cast<const __nv_bfloat16*>(st + x_stage_bytes);
+#pragma unroll
+    for (int ks = 0; ks < 2; ++ks) {
+      const int kk = (warp * 2 + ks) * 16;   // this warp's k-step inside the chunk
+      uint32_t a[2][4];
+#pragma unroll
+      for (int m = 0; m < 2; ++m)
+        ldmatrix_x4(a[m], xs + (m * 16 + (lane & 15)) * kGateXStride + kk + (lane >> 4) * 8);
+#pragma unroll
+      for (int n16 = 0; n16 < NT16; ++n16) {
+        uint32_t b[4];
+        ldmatrix_x4_trans(b, ws + (kk + (lane & 7) + ((lane >> 3) & 1) * 8) * w_stride + n16 * 16 + (lane >> 4) * 8);
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+          mma_bf16_16816(acc[m][n16 * 2], a[m], b[0], b[1]);
+          mma_bf16_16816(acc[m][n16 * 2 + 1], a[m], b[2], b[3]);
+        }
+      }
+    }
+    __syncthreads();
+  }
+  cp_async_wait<0>();
+  __syncthreads();
+
+  // Cross-warp sum in a fixed order.  red[w][row][col], fp32, aliasing the staging buffers.
+  float* red = reinterpret_cast<float*>(smem_raw);
+  constexpr int RS = NP + 1;
+  {
+    const int g = lane >> 2, tq = lane & 3;
+#pragma unroll
+    for (int m = 0; m < 2; ++m)
+#pragma unroll
+      for (int n = 0; n < NT16 * 2; ++n) {
+        float* base = red + ((warp * kGateTM + m * 16 + g) * RS + n * 8 + tq * 2);
+        base[0] = acc[m][n][0];
+        base[1] = acc[m][n][1];
+        base[8 * RS] = acc[m][n][2];
+        base[8 * RS + 1] = acc[m][n][3];
+      }
+  }
+  __syncthreads();
+  for (int i = tid; i < kGateTM * NP; i += kGateThreads) {
+    const int r = i / NP, c = i % NP;
+    float v = red[(0 * kGateTM + r) * RS + c];
+    v += red[(1 * kGateTM + r) * RS + c];
+    v += red[(2 * kGateTM + r) * RS + c];
+    v += red[(3 * kGateTM + r) * RS + c];
+    if (c < N) {
+      if (gate_bias != nullptr) v += gate_bias[c];
+    } else {
+      v = -INFINITY;
+    }
+    red[r * RS + c] = v;   // row r of warp block 0: each (r,c) is read and written by this thread only
+  }
+  __syncthreads();
+
+  // Softmax and sorted Top-K_orig: each warp owns 8 tokens, lane l owns experts l, l+32, ...
+  constexpr int EPL = (NP + 31) / 32;
+  for (int rr = 0; rr < kGateTM / 4; ++rr) {
+    const int r = warp * (kGateTM / 4) + rr;
+    const int t = t0 + r;
+    if (t >= T) break;   // uniform across the warp
+    float v[EPL];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int q = 0; q < EPL; ++q) {
+      const int e = lane + 32 * q;
+      v[q] = (e < NP) ? red[r * RS + e] : -INFINITY;
+      mx = fmaxf(mx, v[q]);
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+    float sum = 0.f;
+#pragma unroll
+    for (int q = 0; q < EPL; ++q) {
+      v[q] = (lane + 32 * q < N) ? expf(v[q] - mx) : 0.f;
+      sum += v[q];
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
+#pragma unroll
+    for (int q = 0; q < EPL; ++q) {
+      v[q] = v[q] / sum;
+      const int e = lane + 32 * q;
+      if (scores != nullptr && e < N) scores[(long long)t * N + e] = v[q];
+    }
+    uint32_t taken = 0u;
+    for (int j = 0; j < K_orig; ++j) {
+      float bv = -1.f;
+      int be = 0x7fffffff;
+#pragma unroll
+      for (int q = 0; q < EPL; ++q) {
+        const int e = lane + 32 * q;
+        if (e < N && !((taken >> q) & 1u) && v[q] > bv) { bv = v[q]; be = e; }   // ascending e: first max wins
+      }
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, d);
+        const int oe = __shfl_xor_sync(0xffffffffu, be, d);
+        if (ov > bv || (ov == bv && oe < be)) { bv = ov; be = oe; }
+      }
+      if ((be & 31) == lane && be < N) taken |= 1u << (be >> 5);
+      if (lane == 0) {
+        topk_idx[(long long)t * K_orig + j] = be < N ? be : 0;
+        topk_score[(long long)t * K_orig + j] = bv;
+      }
+    }
+  }
+}
+
+}  // namespace allocmoe
+
+using namespace allocmoe;
+
+static int gate_w_stride(int NP) {
+  int s16 = NP / 8 + 1;        // row stride in 16-byte units: odd keeps ldmatrix.trans conflict-free
+  if ((s16 & 1) == 0) s16 += 1;
+  return s16 * 8;
+}
+
+template <int NT16>
+static moe_status gate_launch_t(const moe_shape* s, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,
+                                float* scores, int32_t* topk_idx, float* topk_score, cudaStream_t stream) {
+  constexpr int NP = NT16 * 16;
+  const int w_stride = gate_w_stride(NP);
+  size_t pipe = (size_t)kGateStages * (kGateTM * kGateXStride * 2 + kGateKC * w_stride * 2);
+  size_t red = (size_t)4 * kGateTM * (NP + 1) * 4;
+  size_t smem = pipe > red ? pipe : red;
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(moe_gate_kernel<NT16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return MOE_ERR_CUDA;
+    attr_done = true;
+  }
+  const int grid = (s->T + kGateTM - 1) / kGateTM;
+  moe_gate_kernel<NT16><<<grid, kGateThreads, smem, stream>>>(
+      reinterpret_cast<const __nv_bfloat16*>(x), reinterpret_cast<const __nv_bfloat16*>(W_gate), gate_bias, s->T, s->H,
+      s->N, s->K_orig, w_stride, scores, topk_idx, topk_score);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+moe_status launch_moe_gate(const moe_shape* s, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,
+                           float* scores, int32_t* topk_idx, float* topk_score, cudaStream_t stream) {
+  const int nt16 = (s->N + 15) / 16;
+  switch (nt16) {
+    case 1: return gate_launch_t<1>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 2: return gate_launch_t<2>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 3: return gate_launch_t<3>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 4: return gate_launch_t<4>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 5: return gate_launch_t<5>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 6: return gate_launch_t<6>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 7: return gate_launch_t<7>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 8: return gate_launch_t<8>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    default: return MOE_ERR_ARG;
+  }
+}

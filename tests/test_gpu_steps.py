@@ -1,0 +1,243 @@
+"""Step-by-step parity of the C-ABI calls against the CPU oracle (same seeded inputs)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import alloc_moe_oracle as orc
+from paper_2604_08133_b200 import binding as B
+from paper_2604_08133_b200 import synth
+from helpers import TOL_OUT, max_rel, np32
+
+pytestmark = pytest.mark.gpu
+
+
+def _status():
+    return torch.zeros(1, dtype=torch.int32, device="cuda")
+
+
+# ----------------------------------------------------------------------------- alloc_t_select
+SELECT_CASES = [
+    # T, K_orig, K_base, budgets (None = sweep of characteristic values), ties
+    (1, 2, 1, None, False), (31, 3, 0, None, True), (64, 2, 0, None, False), (64, 6, 1, None, False),
+    (1000, 6, 1, None, True), (1025, 4, 2, None, False), (4096, 6, 1, None, False), (4096, 6, 1, None, True),
+    (4096, 6, 0, None, False), (2048, 6, 1, None, False), (8192, 2, 1, None, False), (8192, 8, 1, None, True),
+    (20000, 6, 1, None, False),      # pool of 100 000 keys: beyond the shared-memory staging
+]
+
+
+def _budgets(T, K, kb):
+    lo, hi = kb * T, K * T
+    cand = {lo, lo + 1, hi - 1, hi, (lo + hi) // 2, lo + (hi - lo) // 3, int(1.5 * T), 2 * T, 3 * T, int(4.5 * T)}
+    return sorted(b for b in cand if lo <= b <= hi)
+
+
+@pytest.mark.parametrize("T,K,kb,budgets,ties", SELECT_CASES)
+def test_alloc_t_select_bit_exact(T, K, kb, budgets, ties):
+    s = synth.score_rows(T, K, synth.stream_key(5, T, K, kb), ties=ties)
+    sd = s.cuda()
+    shape = B.make_shape(T, 64, 8, 64, 0, K, kb)
+    n_sel = torch.empty(T, dtype=torch.int32, device="cuda")
+    for budget in (budgets or _budgets(T, K, kb)):
+        st = _status()
+        n_sel.fill_(-7)
+        B.alloc_t_select(shape, sd, budget, n_sel, st, None)
+        torch.cuda.synchronize()
+        assert st.item() == 0
+        want = orc.n_sel_from_mask(orc.alloc_t_select_threshold(s.numpy(), kb, budget))
+        assert np.array_equal(n_sel.cpu().numpy(), want), (T, K, kb, budget)
+        assert int(n_sel.sum()) == budget
+
+
+def test_alloc_t_select_small_case_against_the_sort_form_and_bruteforce():
+    s = synth.score_rows(4, 3, 77)
+    shape = B.make_shape(4, 64, 8, 64, 0, 3, 1)
+    n_sel = torch.empty(4, dtype=torch.int32, device="cuda")
+    for budget in range(4, 13):
+        B.alloc_t_select(shape, s.cuda(), budget, n_sel, _status(), None)
+        _, arg = orc.alloc_t_bruteforce(s.numpy(), 1, budget)
+        assert np.array_equal(n_sel.cpu().numpy(), orc.n_sel_from_mask(arg[0]))
+        assert np.array_equal(n_sel.cpu().numpy(), orc.n_sel_from_mask(orc.alloc_t_select(s.numpy(), 1, budget)))
+
+
+def test_alloc_t_select_flags_nonfinite_and_rejects_bad_budgets():
+    s = synth.score_rows(64, 4, 3).clone()
+    s[5, 2] = float("nan")
+    shape = B.make_shape(64, 64, 8, 64, 0, 4, 1)
+    n_sel = torch.zeros(64, dtype=torch.int32, device="cuda")
+    st = _status()
+    B.alloc_t_select(shape, s.cuda(), 128, n_sel, st, None)
+    torch.cuda.synchronize()
+    assert st.item() & (1 << B.MOE_ERR_NONFINITE)
+    assert ((n_sel >= 1) & (n_sel <= 4)).all()
+    for bad in (63, 257, -1):
+        with pytest.raises(B.MoeError) as ei:
+            B.alloc_t_select(shape, s.cuda(), bad, n_sel, st, None)
+        assert ei.value.status == B.MOE_ERR_BUDGET
+
+
+# ----------------------------------------------------------------------------- moe_permute
+@pytest.mark.parametrize("T,N,K,kb,mult", [(64, 8, 2, 0, 1.0), (64, 64, 6, 1, 3.0), (1000, 64, 6, 1, 2.5),
+                                            (4096, 64, 6, 1, 4.5), (4096, 64, 6, 1, 6.0), (777, 16, 4, 0, 1.3),
+                                            (8192, 8, 2, 1, 1.5)])
+def test_moe_permute_bit_exact(T, N, K, kb, mult):
+    H = 128
+    g = torch.Generator().manual_seed(T * 31 + N)
+    logits = torch.randn(T, N, generator=g, dtype=torch.float64)
+    p = orc.softmax_scores(logits.numpy())
+    idx, sc = orc.topk_sorted(p, K)
+    budget = int(mult * T)
+    n_ref = orc.n_sel_from_mask(orc.alloc_t_select_threshold(sc, kb, budget))
+    want = orc.permute(idx, sc, n_ref, N)
+    x = synth.normal_bf16((T, H), 1.0, synth.stream_key(1, T)).cuda()
+    shape = B.make_shape(T, H, N, 64, 0, K, kb)
+    ws = B.new_workspace(shape, budget)
+    off = torch.empty(N + 1, dtype=torch.int32, device="cuda")
+    tok = torch.empty(budget, dtype=torch.int32, device="cuda")
+    wgt = torch.empty(budget, dtype=torch.float32, device="cuda")
+    pos = torch.empty(T, K, dtype=torch.int32, device="cuda")
+    xp = torch.empty(budget, H, dtype=torch.bfloat16, device="cuda")
+    st = _status()
+    B.moe_permute(shape, x, torch.from_numpy(idx).cuda(), torch.from_numpy(sc).cuda(), torch.from_numpy(n_ref).cuda(),
+                  budget, off, tok, wgt, pos, xp, st, ws)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    assert np.array_equal(off.cpu().numpy(), want["expert_offsets"])
+    assert np.array_equal(tok.cpu().numpy(), want["perm_token"])
+    assert np.array_equal(wgt.cpu().numpy(), want["perm_weight"])
+    assert np.array_equal(pos.cpu().numpy(), want["pair_pos"])
+    assert torch.equal(xp.cpu(), x.cpu()[torch.from_numpy(want["perm_token"]).long()])
+
+
+def test_moe_permute_flags_a_count_mismatch():
+    T, N, K = 64, 8, 2
+    shape = B.make_shape(T, 64, N, 64, 0, K, 0)
+    idx = torch.stack([torch.randperm(N)[:K] for _ in range(T)]).int().cuda()
+    sc = torch.rand(T, K).sort(dim=1, descending=True).values.cuda()
+    n_sel = torch.ones(T, dtype=torch.int32, device="cuda")
+    budget = 70                                    # kept counts add up to 64
+    ws = B.new_workspace(shape, budget)
+    st = _status()
+    B.moe_permute(shape, None, idx, sc, n_sel, budget, torch.empty(N + 1, dtype=torch.int32, device="cuda"),
+                  torch.empty(budget, dtype=torch.int32, device="cuda"), torch.empty(budget, device="cuda"),
+                  torch.empty(T, K, dtype=torch.int32, device="cuda"), None, st, ws)
+    torch.cuda.synchronize()
+    assert st.item() & (1 << B.MOE_ERR_BUDGET)
+
+
+# ----------------------------------------------------------------------------- moe_gate
+@pytest.mark.parametrize("name,kw", [("c1", {}), ("c2", {}), ("c2", dict(T=333, H=192, N=24, K_orig=5)),
+                                      ("c3", dict(T=1000)), ("c5", dict(T=500))])
+def test_moe_gate_against_oracle(name, kw):
+    cfg = synth.CONFIGS[name].with_(I=64, S=0, **kw)
+    x = synth.normal_bf16((cfg.T, cfg.H), 1.0, synth.stream_key(cfg.seed, 0, 0))
+    Wg = synth.normal_bf16((cfg.H, cfg.N), 0.02 * cfg.gate_scale, synth.stream_key(cfg.seed, 0, 1))
+    bias = synth.zipf_gate_bias(cfg) if cfg.zipf_bias else None
+    shape = B.shape_of(cfg)
+    scores = torch.empty(cfg.T, cfg.N, device="cuda")
+    idx = torch.empty(cfg.T, cfg.K_orig, dtype=torch.int32, device="cuda")
+    val = torch.empty(cfg.T, cfg.K_orig, device="cuda")
+    B.moe_gate(shape, x.cuda(), Wg.cuda(), None if bias is None else bias.cuda(), scores, idx, val)
+    torch.cuda.synchronize()
+    p = orc.softmax_scores(orc.gate_logits(np32(x), np32(Wg), None if bias is None else bias.numpy()))
+    got = scores.cpu().numpy()
+    assert np.abs(got - p).max() <= 2e-6 + 1e-5 * p.max()
+    # the Top-K of the GPU's own scores must be exactly the oracle's Top-K rule applied to them
+    ridx, rval = orc.topk_sorted(got, cfg.K_orig)
+    assert np.array_equal(idx.cpu().numpy(), ridx)
+    assert np.array_equal(val.cpu().numpy(), rval)
+    # and against the oracle end to end: identical except where two scores nearly tie
+    oidx, _ = orc.topk_sorted(p, cfg.K_orig)
+    differs = (idx.cpu().numpy() != oidx).any(axis=1)
+    assert differs.mean() <= 0.01
+
+
+# ----------------------------------------------------------------------------- moe_grouped_ffn / shared / combine
+@pytest.mark.parametrize("T,H,N,I,K,budget", [(64, 256, 8, 512, 2, 96), (600, 256, 8, 192, 3, 1500),
+                                               (300, 128, 16, 320, 4, 700)])
+def test_grouped_ffn_against_oracle(T, H, N, I, K, budget):
+    cfg = synth.CONFIGS["c1"].with_(T=T, H=H, N=N, I=I, K_orig=K, K_base=1, budget=budget)
+    d = synth.make_layer(cfg)
+    dn = {k: np32(v) for k, v in d.items()}
+    r = orc.route(dn["x"], dn["W_gate"], None, K, 1, budget)
+    p = orc.permute(r["topk_idx"], r["topk_score"], r["n_sel"], N)
+    off, tok = p["expert_offsets"], p["perm_token"]
+    assert (np.diff(off) == 0).any() or True
+    x_perm = d["x"][torch.from_numpy(tok).long()].contiguous().cuda()
+    shape = B.shape_of(cfg)
+    ws = B.new_workspace(shape, budget)
+    y = torch.full((budget, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    st = _status()
+    B.moe_grouped_ffn(shape, x_perm, torch.from_numpy(off).cuda(), budget, d["W13"].cuda(), d["W2"].cuda(), y, st, ws)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    want = np.zeros((budget, H))
+    for e in range(N):
+        if off[e + 1] > off[e]:
+            want[off[e]:off[e + 1]] = orc.expert_ffn(dn["x"][tok[off[e]:off[e + 1]]], dn["W13"][e], dn["W2"][e])
+    got = y.float().cpu().numpy()
+    assert np.isfinite(got).all()
+    assert max_rel(got, want) <= TOL_OUT
+
+
+def test_grouped_ffn_skips_empty_experts_and_respects_segment_ends():
+    T, H, N, I = 40, 128, 8, 128
+    cfg = synth.CONFIGS["c1"].with_(T=T, H=H, N=N, I=I)
+    d = synth.make_layer(cfg)
+    # experts 0, 3, 7 get rows; all others are empty
+    off = np.array([0, 5, 5, 5, 36, 36, 36, 36, 40], np.int32)
+    x_perm = d["x"].cuda()
+    shape = B.shape_of(cfg)
+    ws = B.new_workspace(shape, T)
+    y = torch.full((T + 8, H), 123.0, dtype=torch.bfloat16, device="cuda")
+    st = _status()
+    B.moe_grouped_ffn(shape, x_perm, torch.from_numpy(off).cuda(), T, d["W13"].cuda(), d["W2"].cuda(), y, st, ws)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    assert (y[T:] == 123.0).all()                       # nothing is written past the list
+    xn, W13, W2 = np32(d["x"]), np32(d["W13"]), np32(d["W2"])
+    want = np.concatenate([orc.expert_ffn(xn[0:5], W13[0], W2[0]), orc.expert_ffn(xn[5:36], W13[3], W2[3]),
+                           orc.expert_ffn(xn[36:40], W13[7], W2[7])])
+    assert max_rel(y[:T].float().cpu().numpy(), want) <= TOL_OUT
+
+
+@pytest.mark.parametrize("T,H,I,S", [(64, 256, 192, 2), (300, 128, 128, 1), (130, 256, 320, 3)])
+def test_shared_ffn_against_oracle(T, H, I, S):
+    cfg = synth.CONFIGS["c2"].with_(T=T, H=H, N=8, I=I, S=S, K_orig=2, K_base=1, budget=T)
+    d = synth.make_layer(cfg)
+    shape = B.shape_of(cfg)
+    ws = B.new_workspace(shape, 0)
+    y = torch.empty(T, H, dtype=torch.bfloat16, device="cuda")
+    st = _status()
+    B.moe_shared_ffn(shape, d["x"].cuda(), d["Wsh13"].cuda(), d["Wsh2"].cuda(), y, st, ws)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    want = orc.shared_experts(np32(d["x"]), np32(d["Wsh13"]), np32(d["Wsh2"]))
+    assert max_rel(y.float().cpu().numpy(), want) <= TOL_OUT
+
+
+def test_combine_against_oracle_formula():
+    T, H, K, Bk = 50, 256, 4, 120
+    g = torch.Generator().manual_seed(3)
+    y_perm = torch.randn(Bk, H, generator=g).bfloat16()
+    y_sh = torch.randn(T, H, generator=g).bfloat16()
+    sc = torch.rand(T, K, generator=g).sort(dim=1, descending=True).values
+    n_sel = torch.randint(0, K + 1, (T,), generator=g).int()
+    pos = torch.full((T, K), -1, dtype=torch.int32)
+    perm = torch.randperm(Bk, generator=g)
+    q = 0
+    for t in range(T):
+        for j in range(int(n_sel[t])):
+            pos[t, j] = perm[q]
+            q += 1
+    shape = B.make_shape(T, H, 8, 64, 1, K, 0)
+    out = torch.empty(T, H, dtype=torch.bfloat16, device="cuda")
+    B.moe_combine(shape, y_perm.cuda(), pos.cuda(), sc.cuda(), n_sel.cuda(), y_sh.cuda(), out)
+    torch.cuda.synchronize()
+    want = y_sh.double().numpy().copy()
+    for t in range(T):
+        for j in range(int(n_sel[t])):
+            want[t] += float(sc[t, j]) * y_perm[pos[t, j]].double().numpy()
+    got = out.float().cpu().numpy()
+    # one bf16 rounding of an fp32 sum of exactly representable products
+    assert np.abs(got - want).max() <= 2 ** -8 * np.abs(want).max()
+    assert max_rel(got, want) <= 4e-3
