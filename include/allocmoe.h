@@ -131,13 +131,19 @@ moe_status moe_combine(const moe_shape* shape, const uint16_t* y_perm, const int
 
 /* The whole layer on one stream: moe_gate, alloc_t_select, moe_permute, moe_grouped_ffn
  * (+ moe_shared_ffn when S > 0), moe_combine; all intermediates live in `ws`.
- * Wsh13 / Wsh2 are ignored when S == 0.  With residual != 0 the layer input is added:
- * out = x + MoE(x) (fp32 add, one bf16 rounding), the step of a residual layer stack. */
+ * Wsh13 / Wsh2 are ignored when S == 0.
+ *   residual  device bf16 [T,H] or NULL: added to the result, out = residual + MoE(x) (fp32 add,
+ *             one bf16 rounding): the step of a residual layer stack.  May alias x, not out. */
 moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const uint16_t* W_gate,
                              const float* gate_bias, const uint16_t* W13, const uint16_t* W2,
                              const uint16_t* Wsh13, const uint16_t* Wsh2, int64_t budget,
-                             int32_t residual, uint16_t* out, int32_t* dev_status, void* ws,
+                             const uint16_t* residual, uint16_t* out, int32_t* dev_status, void* ws,
                              size_t ws_bytes, void* stream);
+
+/* Pre-norm of a residual layer stack (not part of the paper's method; the layer stack workload
+ * needs it, see the stack recurrence x_{l+1} = x_l + MoE(norm(x_l))): out[t] = x[t] / sqrt(mean_h
+ * x[t,h]^2 + 1e-6), unit gain, fp32 math, one bf16 rounding.  x, out device bf16 [T,H]. */
+moe_status moe_rmsnorm(const moe_shape* shape, const uint16_t* x, uint16_t* out, void* stream);
 
 /* Device addresses of the routing intermediates that moe_layer_forward, called with this shape,
  * this budget and this workspace, leaves in `ws` (for inspection and tests; valid until ws is
@@ -146,6 +152,15 @@ moe_status moe_layer_intermediates(const moe_shape* shape, int64_t budget, void*
                                    size_t ws_bytes, int32_t** topk_idx, float** topk_score,
                                    int32_t** n_sel, int32_t** expert_offsets,
                                    int32_t** perm_token, int32_t** pair_pos, uint16_t** y_perm);
+
+/* Instrumentation (no counterpart in the paper): with profiling on, moe_layer_forward records
+ * CUDA events at its stage boundaries; moe_profile_read waits for the last forward call and
+ * returns the device time in milliseconds of its 6 stages: gate, alloc_t_select, moe_permute,
+ * expert GEMM-1 (with SwiGLU), expert GEMM-2, combine.  Host-side state only (events); one
+ * forward call at a time may be in flight while profiling.  Off by default. */
+#define MOE_PROFILE_STAGES 6
+moe_status moe_profile_enable(int32_t on);
+moe_status moe_profile_read(float* stage_ms /* host [MOE_PROFILE_STAGES] */);
 
 #ifdef __cplusplus
 }

@@ -285,14 +285,25 @@ def bf16_round(a) -> np.ndarray:
     return f
 
 
+def rmsnorm(x, eps: float = 1e-6) -> np.ndarray:
+    """x[t] / sqrt(mean_h x[t,h]^2 + eps), unit gain, fp64 (the pre-norm of the layer stack)."""
+    xx = np.asarray(x, F64)
+    return xx / np.sqrt((xx * xx).mean(axis=1, keepdims=True) + eps)
+
+
 def stack_forward(x0, layers: Sequence[Dict[str, np.ndarray]], K_orig: int, K_base: int,
-                  budgets: Sequence[int]) -> List[np.ndarray]:
-    """Residual stack x_{l+1} = x_l + MoE_l(x_l) with the stream stored in bf16 between
-    layers (storage format of the workload).  Returns [x_1, ..., x_L] as fp32 arrays."""
+                  budgets: Sequence[int], prenorm: bool = True) -> List[np.ndarray]:
+    """Residual stack with the stream stored in bf16 between layers (storage format of the
+    workload): x_{l+1} = x_l + MoE_l(norm(x_l)), norm = RMS normalisation rounded to bf16, or the
+    identity with prenorm=False.  The literal recurrence x + MoE(x) squares the stream's scale
+    every layer (SwiGLU is quadratic in its input) and overflows within a dozen layers, so the
+    stack workload is run pre-norm, as the transformer blocks it stands for are.
+    Returns [x_1, ..., x_L] as fp32 arrays."""
     xs = []
     x = np.asarray(x0, np.float32)
     for lw, b in zip(layers, budgets):
-        out = layer_forward(x, lw["W_gate"], lw.get("gate_bias"), lw["W13"], lw["W2"],
+        xin = bf16_round(rmsnorm(x)) if prenorm else x
+        out = layer_forward(xin, lw["W_gate"], lw.get("gate_bias"), lw["W13"], lw["W2"],
                             lw.get("Wsh13"), lw.get("Wsh2"), K_orig, K_base, b)["out"]
         x = bf16_round(np.asarray(x, F64) + out)
         xs.append(x)

@@ -15,7 +15,9 @@ LIB_PATH = os.path.join(_PKG, "liballocmoe.so")
 MOE_OK, MOE_ERR_ARG, MOE_ERR_BUDGET, MOE_ERR_WORKSPACE, MOE_ERR_CUDA, MOE_ERR_NONFINITE, MOE_ERR_TIMEOUT = range(7)
 
 EXPORTS = ("moe_status_string", "moe_workspace_bytes", "moe_gate", "alloc_t_select", "moe_permute",
-           "moe_grouped_ffn", "moe_shared_ffn", "moe_combine", "moe_layer_forward", "moe_layer_intermediates")
+           "moe_grouped_ffn", "moe_shared_ffn", "moe_combine", "moe_layer_forward", "moe_layer_intermediates",
+           "moe_rmsnorm", "moe_profile_enable", "moe_profile_read")
+PROFILE_STAGES = ("gate", "select", "permute", "ffn_gemm1", "ffn_gemm2", "combine")
 
 
 class MoeShape(ctypes.Structure):
@@ -54,8 +56,11 @@ def lib() -> ctypes.CDLL:
             "moe_grouped_ffn": [sp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp],
             "moe_shared_ffn": [sp, vp, vp, vp, vp, vp, vp, sz, vp],
             "moe_combine": [sp, vp, vp, vp, vp, vp, vp, vp],
-            "moe_layer_forward": [sp, vp, vp, vp, vp, vp, vp, vp, i64, ctypes.c_int32, vp, vp, vp, sz, vp],
+            "moe_layer_forward": [sp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, sz, vp],
+            "moe_rmsnorm": [sp, vp, vp, vp],
             "moe_layer_intermediates": [sp, i64, vp, sz] + [ctypes.POINTER(vp)] * 7,
+            "moe_profile_enable": [ctypes.c_int32],
+            "moe_profile_read": [ctypes.POINTER(ctypes.c_float)],
         }
         for name, argtypes in sigs.items():
             fn = getattr(L, name)
@@ -141,10 +146,14 @@ def moe_combine(shape, y_perm, pair_pos, topk_score, n_sel, y_shared, out, strea
 
 
 def moe_layer_forward(shape, x, W_gate, gate_bias, W13, W2, Wsh13, Wsh2, budget, out, dev_status, ws,
-                      residual: bool = False, stream=None):
+                      residual: Optional[torch.Tensor] = None, stream=None):
     _check("moe_layer_forward", lib().moe_layer_forward(ctypes.byref(shape), _p(x), _p(W_gate), _p(gate_bias), _p(W13),
-                                                        _p(W2), _p(Wsh13), _p(Wsh2), int(budget), int(bool(residual)),
+                                                        _p(W2), _p(Wsh13), _p(Wsh2), int(budget), _p(residual),
                                                         _p(out), _p(dev_status), _p(ws), ws.numel(), _stream(stream)))
+
+
+def moe_rmsnorm(shape, x, out, stream=None):
+    _check("moe_rmsnorm", lib().moe_rmsnorm(ctypes.byref(shape), _p(x), _p(out), _stream(stream)))
 
 
 def moe_layer_intermediates(shape, budget, ws) -> Dict[str, torch.Tensor]:
@@ -168,3 +177,14 @@ def moe_layer_intermediates(shape, budget, ws) -> Dict[str, torch.Tensor]:
         pair_pos=view(ptrs[5], T * K * 4, torch.int32, (T, K)),
         y_perm=view(ptrs[6], B * H * 2, torch.bfloat16, (B, H)),
     )
+
+
+def moe_profile_enable(on: bool):
+    _check("moe_profile_enable", lib().moe_profile_enable(int(bool(on))))
+
+
+def moe_profile_read() -> Dict[str, float]:
+    """Device milliseconds of the six stages of the last moe_layer_forward call."""
+    buf = (ctypes.c_float * len(PROFILE_STAGES))()
+    _check("moe_profile_read", lib().moe_profile_read(buf))
+    return {k: float(buf[i]) for i, k in enumerate(PROFILE_STAGES)}

@@ -12,9 +12,10 @@ moe_status launch_moe_permute(const moe_shape*, const uint16_t*, const int32_t*,
                               int32_t*, int32_t*, float*, int32_t*, uint16_t*, int32_t*, int32_t*, cudaStream_t);
 moe_status launch_ffn(const moe_shape*, const uint16_t*, const int32_t*, int64_t, const uint16_t*, const uint16_t*,
                       uint16_t*, uint16_t*, const uint16_t*, const uint16_t*, const uint16_t*, uint16_t*, uint16_t*,
-                      int32_t*, cudaStream_t);
+                      int32_t*, cudaStream_t, cudaEvent_t);
 moe_status launch_moe_combine(const moe_shape*, const uint16_t*, const int32_t*, const float*, const int32_t*,
                               const uint16_t*, const uint16_t*, long long, uint16_t*, cudaStream_t);
+moe_status launch_rmsnorm(const moe_shape*, const uint16_t*, uint16_t*, cudaStream_t);
 
 namespace {
 
@@ -69,6 +70,14 @@ WsLayout ws_layout(const moe_shape* s, int64_t budget_max) {
 
 template <typename T>
 T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<unsigned char*>(ws) + off); }
+
+// Optional stage timing of moe_layer_forward (off by default): events at the stage boundaries.
+constexpr int kProfStages = 6;   // gate, select, permute, ffn GEMM-1, ffn GEMM-2, combine
+bool g_prof_on = false;
+cudaEvent_t g_prof_ev[kProfStages + 1];
+void prof_mark(int i, cudaStream_t st) {
+  if (g_prof_on) cudaEventRecord(g_prof_ev[i], st);
+}
 
 }  // namespace
 
@@ -134,7 +143,7 @@ moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_perm, const
   const WsLayout L = ws_layout(shape, budget);
   if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
   return launch_ffn(shape, x_perm, expert_offsets, budget, W13, W2, at<uint16_t>(ws, L.h), y_perm, nullptr, nullptr,
-                    nullptr, nullptr, nullptr, dev_status, (cudaStream_t)stream);
+                    nullptr, nullptr, nullptr, dev_status, (cudaStream_t)stream, nullptr);
 }
 
 moe_status moe_shared_ffn(const moe_shape* shape, const uint16_t* x, const uint16_t* Wsh13, const uint16_t* Wsh2,
@@ -144,7 +153,7 @@ moe_status moe_shared_ffn(const moe_shape* shape, const uint16_t* x, const uint1
   const WsLayout L = ws_layout(shape, 0);
   if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
   return launch_ffn(shape, nullptr, nullptr, 0, nullptr, nullptr, nullptr, nullptr, x, Wsh13, Wsh2,
-                    at<uint16_t>(ws, L.h_sh), y_shared, dev_status, (cudaStream_t)stream);
+                    at<uint16_t>(ws, L.h_sh), y_shared, dev_status, (cudaStream_t)stream, nullptr);
 }
 
 moe_status moe_combine(const moe_shape* shape, const uint16_t* y_perm, const int32_t* pair_pos,
@@ -158,13 +167,14 @@ moe_status moe_combine(const moe_shape* shape, const uint16_t* y_perm, const int
 
 moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,
                              const uint16_t* W13, const uint16_t* W2, const uint16_t* Wsh13, const uint16_t* Wsh2,
-                             int64_t budget, int32_t residual, uint16_t* out, int32_t* dev_status, void* ws,
+                             int64_t budget, const uint16_t* residual, uint16_t* out, int32_t* dev_status, void* ws,
                              size_t ws_bytes, void* stream) {
   if (!shape_ok(shape) || !x || !W_gate || !W13 || !W2 || !out || !dev_status || !ws) return MOE_ERR_ARG;
   if (shape->S > 0 && (!Wsh13 || !Wsh2)) return MOE_ERR_ARG;
   if (!aligned16(x) || !aligned16(W_gate) || !aligned16(W13) || !aligned16(W2) || !aligned16(out) || !aligned16(ws))
     return MOE_ERR_ARG;
   if (shape->S > 0 && (!aligned16(Wsh13) || !aligned16(Wsh2))) return MOE_ERR_ARG;
+  if (residual != nullptr && (!aligned16(residual) || residual == out)) return MOE_ERR_ARG;
   if (!budget_ok(shape, budget)) return MOE_ERR_BUDGET;
   const WsLayout L = ws_layout(shape, budget);
   if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
@@ -180,18 +190,51 @@ moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const ui
   uint16_t* y_perm = at<uint16_t>(ws, L.y_perm);
   uint16_t* y_shared = shape->S > 0 ? at<uint16_t>(ws, L.y_shared) : nullptr;
 
+  prof_mark(0, st);
   moe_status r = launch_moe_gate(shape, x, W_gate, gate_bias, nullptr, topk_idx, topk_score, st);
   if (r != MOE_OK) return r;
+  prof_mark(1, st);
   r = launch_alloc_t_select(shape, topk_score, budget, n_sel, dev_status, st);
   if (r != MOE_OK) return r;
+  prof_mark(2, st);
   r = launch_moe_permute(shape, x, topk_idx, topk_score, n_sel, budget, expert_offsets, perm_token, perm_weight,
                          pair_pos, x_perm, dev_status, at<int32_t>(ws, L.seg_counts), st);
   if (r != MOE_OK) return r;
+  prof_mark(3, st);
   r = launch_ffn(shape, x_perm, expert_offsets, budget, W13, W2, at<uint16_t>(ws, L.h), y_perm,
-                 shape->S > 0 ? x : nullptr, Wsh13, Wsh2, at<uint16_t>(ws, L.h_sh), y_shared, dev_status, st);
+                 shape->S > 0 ? x : nullptr, Wsh13, Wsh2, at<uint16_t>(ws, L.h_sh), y_shared, dev_status, st,
+                 g_prof_on ? g_prof_ev[4] : nullptr);
   if (r != MOE_OK) return r;
-  return launch_moe_combine(shape, y_perm, pair_pos, topk_score, n_sel, y_shared, residual ? x : nullptr, budget, out,
-                            st);
+  prof_mark(5, st);
+  r = launch_moe_combine(shape, y_perm, pair_pos, topk_score, n_sel, y_shared, residual, budget, out,
+                         st);
+  prof_mark(6, st);
+  return r;
+}
+
+moe_status moe_rmsnorm(const moe_shape* shape, const uint16_t* x, uint16_t* out, void* stream) {
+  if (!shape_ok(shape) || !x || !out || !aligned16(x) || !aligned16(out)) return MOE_ERR_ARG;
+  return launch_rmsnorm(shape, x, out, (cudaStream_t)stream);
+}
+
+moe_status moe_profile_enable(int32_t on) {
+  if (on && !g_prof_on) {
+    for (int i = 0; i <= kProfStages; ++i)
+      if (cudaEventCreate(&g_prof_ev[i]) != cudaSuccess) return MOE_ERR_CUDA;
+    g_prof_on = true;
+  } else if (!on && g_prof_on) {
+    g_prof_on = false;
+    for (int i = 0; i <= kProfStages; ++i) cudaEventDestroy(g_prof_ev[i]);
+  }
+  return MOE_OK;
+}
+
+moe_status moe_profile_read(float* stage_ms) {
+  if (!g_prof_on || !stage_ms) return MOE_ERR_ARG;
+  if (cudaEventSynchronize(g_prof_ev[kProfStages]) != cudaSuccess) return MOE_ERR_CUDA;
+  for (int i = 0; i < kProfStages; ++i)
+    if (cudaEventElapsedTime(&stage_ms[i], g_prof_ev[i], g_prof_ev[i + 1]) != cudaSuccess) return MOE_ERR_CUDA;
+  return MOE_OK;
 }
 
 moe_status moe_layer_intermediates(const moe_shape* shape, int64_t budget_max, void* ws, size_t ws_bytes,

@@ -57,9 +57,55 @@ combine_kernel(const uint4* __restrict__ y_perm, const int32_t* __restrict__ pai
   }
 }
 
+// Pre-norm of the layer stack: out[t] = x[t] * rsqrt(mean(x[t]^2) + eps).  One CTA per token; the
+// sum of squares is reduced in a fixed order (lanes by shuffle, warps in index order).
+__global__ void __launch_bounds__(256)
+rmsnorm_kernel(const uint4* __restrict__ x, int row_vec, int H, uint4* __restrict__ out) {
+  __shared__ float warp_part[8];
+  __shared__ float s_scale;
+  const int t = blockIdx.x;
+  float ss = 0.f;
+  for (int c = threadIdx.x; c < row_vec; c += blockDim.x) {
+    const uint4 v = __ldg(x + (long long)t * row_vec + c);
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float a = bf16_bits_to_float(u[q] & 0xFFFFu), b = bf16_bits_to_float(u[q] >> 16);
+      ss = fmaf(a, a, ss);
+      ss = fmaf(b, b, ss);
+    }
+  }
+#pragma unroll
+  for (int d = 16; d >= 1; d >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
+  if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float tot = 0.f;
+    for (int w = 0; w < 8; ++w) tot += warp_part[w];
+    s_scale = rsqrtf(tot / (float)H + 1e-6f);
+  }
+  __syncthreads();
+  const float sc = s_scale;
+  for (int c = threadIdx.x; c < row_vec; c += blockDim.x) {
+    const uint4 v = __ldg(x + (long long)t * row_vec + c);
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      o[q] = pack_bf16x2(bf16_bits_to_float(u[q] & 0xFFFFu) * sc, bf16_bits_to_float(u[q] >> 16) * sc);
+    out[(long long)t * row_vec + c] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
 }  // namespace allocmoe
 
 using namespace allocmoe;
+
+moe_status launch_rmsnorm(const moe_shape* s, const uint16_t* x, uint16_t* out, cudaStream_t stream) {
+  rmsnorm_kernel<<<s->T, 256, 0, stream>>>(reinterpret_cast<const uint4*>(x), s->H / 8, s->H,
+                                           reinterpret_cast<uint4*>(out));
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
 
 moe_status launch_moe_combine(const moe_shape* s, const uint16_t* y_perm, const int32_t* pair_pos,
                               const float* topk_score, const int32_t* n_sel, const uint16_t* y_shared,

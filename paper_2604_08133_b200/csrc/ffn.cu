@@ -378,7 +378,7 @@ static moe_status launch_gemm(const FfnGemmParams& p, const CUtensorMap& ar, con
 moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t* expert_offsets, int64_t budget,
                       const uint16_t* W13, const uint16_t* W2, uint16_t* h, uint16_t* y_perm, const uint16_t* x_shared,
                       const uint16_t* Wsh13, const uint16_t* Wsh2, uint16_t* h_sh, uint16_t* y_shared,
-                      int32_t* dev_status, cudaStream_t stream) {
+                      int32_t* dev_status, cudaStream_t stream, cudaEvent_t between) {
   const bool routed = (budget > 0 && x_perm != nullptr);
   const bool shared = (s->S > 0 && x_shared != nullptr);
   if (!routed && !shared) return MOE_OK;
@@ -418,6 +418,7 @@ moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t*
   p.ld_out_shared = (long long)s->S * s->I;
   moe_status st = launch_gemm<true>(p, a1r, b1r, a1s, b1s, stream);
   if (st != MOE_OK) return st;
+  if (between != nullptr) cudaEventRecord(between, stream);
   // GEMM-2
   p.n_per_sub = s->H;
   p.k_per_sub = s->I;

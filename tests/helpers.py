@@ -23,7 +23,7 @@ def dev_layer(cfg, layer=0, with_x=True):
     return synth.make_layer(cfg, layer, device="cuda", with_x=with_x)
 
 
-def forward_gpu(cfg, d, budget=None, residual=False, x=None):
+def forward_gpu(cfg, d, budget=None, residual=None, x=None):
     """One moe_layer_forward call; returns (out bf16 [T,H], intermediates dict, dev_status int)."""
     budget = cfg.budget if budget is None else budget
     shape = B.shape_of(cfg)

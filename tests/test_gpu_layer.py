@@ -1,0 +1,205 @@
+"""Whole-layer parity of moe_layer_forward against the CPU oracle on the five workloads.
+
+Two comparisons (the GPU's fp32 scores differ from the oracle's in the last bits, so a pair whose
+score sits within an ulp or two of the selection threshold may flip):
+  fed   the oracle's Alloc-T, permutation, experts and Eq. 2 run on the GPU's own Top-K scores:
+        selection, offsets and permutation must be bit-exact, outputs within TOL_OUT;
+  free  the oracle runs end to end from x: flipped pairs are counted and must be rare and
+        near-ties; outputs are compared on tokens whose selection is identical.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import alloc_moe_oracle as orc
+from paper_2604_08133_b200 import binding as B
+from paper_2604_08133_b200 import synth
+from helpers import TOL_OUT, check_routing_fed, dev_layer, forward_gpu, max_rel, np32
+
+pytestmark = pytest.mark.gpu
+
+
+def _cpu(d):
+    return {k: np32(v) for k, v in d.items()}
+
+
+def _full_check(cfg, budget=None):
+    budget = cfg.budget if budget is None else budget
+    d = dev_layer(cfg)
+    out, inter, status = forward_gpu(cfg, d, budget)
+    assert status == 0
+    idx, sc, n_ref = check_routing_fed(cfg, inter, budget)
+    dn = _cpu(d)
+    got = out.float().cpu().numpy()
+    # fed: Eq. 2 on the GPU's routing
+    fed = orc.combine(dn["x"], idx, sc, n_ref, dn["W13"], dn["W2"], dn["Wsh13"], dn["Wsh2"])
+    assert max_rel(got, fed) <= TOL_OUT
+    # free: oracle end to end
+    free = orc.layer_forward(dn["x"], dn["W_gate"], dn["gate_bias"], dn["W13"], dn["W2"], dn["Wsh13"], dn["Wsh2"],
+                             cfg.K_orig, cfg.K_base, budget)
+    same = (free["n_sel"] == n_ref) & (free["topk_idx"] == idx).all(axis=1)
+    flips = int((~same).sum())
+    assert flips <= max(1, cfg.T // 100), f"{flips} tokens with a different selection"
+    assert max_rel(got[same], free["out"][same]) <= TOL_OUT
+    return flips
+
+
+def test_c1_degenerate_top1():
+    cfg = synth.CONFIGS["c1"]
+    _full_check(cfg)
+    # K_base = K_l: plain Top-1 routing
+    _, inter, _ = forward_gpu(cfg, dev_layer(cfg))
+    assert (inter["n_sel"] == 1).all()
+
+
+def test_c1_kbase0_redistributes():
+    cfg = synth.CONFIGS["c1k0"]
+    _full_check(cfg)
+    _, inter, _ = forward_gpu(cfg, dev_layer(cfg))
+    n = inter["n_sel"].cpu().numpy()
+    assert n.sum() == 64 and n.min() == 0 and n.max() == 2      # budget moved between tokens
+
+
+def test_c2_decode():
+    cfg = synth.CONFIGS["c2"]
+    _full_check(cfg)
+    _full_check(cfg, budget=6 * cfg.T)       # full Top-K_orig, the unbudgeted layer
+
+
+def test_ragged_multi_tile_layer():
+    # several 128-row tiles per expert with ragged ends, a partial column tile (I=192), S=1
+    cfg = synth.CONFIGS["c2"].with_(T=700, H=256, N=8, I=192, S=1, K_orig=3, K_base=1, budget=1500)
+    _full_check(cfg)
+    cfg = cfg.with_(K_base=0, budget=701)
+    _full_check(cfg)
+
+
+def test_residual_flag_adds_the_input():
+    cfg = synth.CONFIGS["c1k0"]
+    d = dev_layer(cfg)
+    out0, _, _ = forward_gpu(cfg, d)
+    out1, inter, _ = forward_gpu(cfg, d, residual=d["x"])
+    dn = _cpu(d)
+    ref = orc.combine(dn["x"], inter["topk_idx"].cpu().numpy(), inter["topk_score"].cpu().numpy(),
+                      inter["n_sel"].cpu().numpy(), dn["W13"], dn["W2"]) + dn["x"].astype(np.float64)
+    assert max_rel(out1.float().cpu().numpy(), ref) <= 4e-3
+    assert not torch.equal(out0, out1)
+
+
+def test_forward_is_deterministic():
+    cfg = synth.CONFIGS["c2"]
+    d = dev_layer(cfg)
+    a, ia, _ = forward_gpu(cfg, d)
+    for _ in range(5):
+        b, ib, _ = forward_gpu(cfg, d)
+        assert torch.equal(a, b)
+        assert torch.equal(ia["perm_token"], ib["perm_token"])
+
+
+def test_host_checked_errors_launch_nothing():
+    cfg = synth.CONFIGS["c1"]
+    d = dev_layer(cfg)
+    shape = B.shape_of(cfg)
+    ws = B.new_workspace(shape, cfg.K_orig * cfg.T)
+    out = torch.full_like(d["x"], 7.0)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    args = (d["x"], d["W_gate"], None, d["W13"], d["W2"], None, None)
+    for budget, want in ((cfg.T - 1, B.MOE_ERR_BUDGET), (cfg.K_orig * cfg.T + 1, B.MOE_ERR_BUDGET)):
+        with pytest.raises(B.MoeError) as ei:
+            B.moe_layer_forward(shape, *args, budget, out, st, ws)
+        assert ei.value.status == want
+    with pytest.raises(B.MoeError) as ei:
+        B.moe_layer_forward(shape, *args, cfg.budget, out, st, ws[:1024])
+    assert ei.value.status == B.MOE_ERR_WORKSPACE
+    bad = B.make_shape(cfg.T, cfg.H + 1, cfg.N, cfg.I, 0, 2, 1)
+    with pytest.raises(B.MoeError) as ei:
+        B.moe_layer_forward(bad, *args, cfg.budget, out, st, ws)
+    assert ei.value.status == B.MOE_ERR_ARG
+    with pytest.raises(B.MoeError) as ei:
+        B.moe_layer_forward(shape, d["x"].view(-1)[1:], *args[1:], cfg.budget, out, st, ws)   # misaligned x
+    assert ei.value.status == B.MOE_ERR_ARG
+    torch.cuda.synchronize()
+    assert (out == 7.0).all() and st.item() == 0
+
+
+# ----------------------------------------------------------------------------- full sizes, sampled rows
+def _sampled_check(cfg, d, budget, rows, x=None, residual=None):
+    out, inter, status = forward_gpu(cfg, d, budget, residual=residual, x=x)
+    assert status == 0
+    idx, sc, n_ref = check_routing_fed(cfg, inter, budget)
+    xin = d["x"] if x is None else x
+    xn = np32(xin)
+    ref = orc.combine(xn, idx, sc, n_ref, np32(d["W13"]), np32(d["W2"]), np32(d["Wsh13"]), np32(d["Wsh2"]), rows=rows)
+    if residual is not None:
+        ref = ref + np32(residual)[rows].astype(np.float64)
+    got = out.float().cpu().numpy()[rows]
+    assert bool(torch.isfinite(out.float()).all())
+    assert max_rel(got, ref) <= TOL_OUT
+    return out, inter
+
+
+def _sample_rows(T, n, key):
+    return sorted(set(synth.permutation(T, synth.stream_key(123, key))[:n]))
+
+
+def test_c3_prefill_full_size_budget_sweep():
+    cfg = synth.CONFIGS["c3"]
+    d = dev_layer(cfg)
+    rows = _sample_rows(cfg.T, 48, 3)
+    touched = []
+    for mult in synth.C3_BUDGET_MULTS:
+        budget = int(mult * cfg.T)
+        _, inter = _sampled_check(cfg, d, budget, rows if mult == 3.0 else rows[:8])
+        off = inter["expert_offsets"].cpu().numpy()
+        assert off[-1] == budget
+        touched.append(int((np.diff(off) > 0).sum()))
+    # free-running comparison of the routing at the paper's half budget
+    dn = {k: np32(d[k]) for k in ("x", "W_gate", "gate_bias")}
+    r = orc.route(dn["x"], dn["W_gate"], dn["gate_bias"], cfg.K_orig, cfg.K_base, 3 * cfg.T)
+    _, inter, _ = forward_gpu(cfg, d, 3 * cfg.T)
+    same = (r["n_sel"] == inter["n_sel"].cpu().numpy()) & (r["topk_idx"] == inter["topk_idx"].cpu().numpy()).all(axis=1)
+    assert (~same).sum() <= cfg.T // 100
+
+
+def test_c5_large_experts_full_size():
+    cfg = synth.CONFIGS["c5"]
+    d = dev_layer(cfg)
+    _sampled_check(cfg, d, cfg.budget, _sample_rows(cfg.T, 12, 5))
+
+
+def test_rmsnorm_against_oracle():
+    cfg = synth.CONFIGS["c4"].with_(T=300)
+    x = (synth.normal_bf16((cfg.T, cfg.H), 3.0, 11).cuda())
+    out = torch.empty_like(x)
+    B.moe_rmsnorm(B.shape_of(cfg), x, out)
+    torch.cuda.synchronize()
+    want = orc.rmsnorm(np32(x))
+    got = out.float().cpu().numpy()
+    assert np.abs(got - want).max() <= 2 ** -8 * np.abs(want).max() * 1.01
+
+
+def test_c4_stack_teacher_forced():
+    """26 layers, per-layer budgets, pre-norm residual stream in bf16:
+    x_{l+1} = x_l + MoE_l(rmsnorm(x_l)).  Every layer's routing is checked in full; outputs of
+    three layers are checked on sampled rows, each against the oracle run on the GPU's own input to
+    that layer (teacher forcing, so errors do not compound)."""
+    cfg = synth.CONFIGS["c4"]
+    ks = synth.stack_budgets(cfg)
+    shape = B.shape_of(cfg)
+    x = synth.make_layer(cfg.with_(N=8, I=64, S=0), 0, device="cuda")["x"]
+    xn = torch.empty_like(x)
+    rows = _sample_rows(cfg.T, 16, 4)
+    for l in range(cfg.n_layers):
+        d = dev_layer(cfg, l, with_x=False)
+        budget = ks[l] * cfg.T
+        B.moe_rmsnorm(shape, x, xn)
+        if l in (0, 12, 25):
+            out, _ = _sampled_check(cfg, d, budget, rows, x=xn, residual=x)
+        else:
+            out, inter, status = forward_gpu(cfg, d, budget, residual=x, x=xn)
+            assert status == 0
+            check_routing_fed(cfg, inter, budget)
+        assert bool(torch.isfinite(out.float()).all())
+        assert 0.5 < float(out.float().std()) < 50.0          # the pre-norm stream grows slowly
+        x = out
+        del d

@@ -137,13 +137,26 @@ def test_stack_is_the_residual_recurrence():
               for l in range(3)]
     budgets = [8, 16, 24]
     xs = orc.stack_forward(layers[0]["x"], layers, cfg.K_orig, cfg.K_base, budgets)
+    xs_literal = orc.stack_forward(layers[0]["x"], layers, cfg.K_orig, cfg.K_base, budgets, prenorm=False)
     x = layers[0]["x"]
     for l in range(3):
         lw = layers[l]
-        o = orc.layer_forward(x, lw["W_gate"], lw["gate_bias"], lw["W13"], lw["W2"], lw["Wsh13"], lw["Wsh2"],
+        xd = torch.from_numpy(x).double()
+        xn = (xd * torch.rsqrt(xd.pow(2).mean(dim=1, keepdim=True) + 1e-6)).to(torch.bfloat16).float().numpy()
+        o = orc.layer_forward(xn, lw["W_gate"], lw["gate_bias"], lw["W13"], lw["W2"], lw["Wsh13"], lw["Wsh2"],
                               cfg.K_orig, cfg.K_base, budgets[l])["out"]
         x = torch.from_numpy((x.astype(np.float64) + o).astype(np.float32)).to(torch.bfloat16).float().numpy()
         assert np.array_equal(xs[l], x)
+    assert not np.array_equal(xs[0], xs_literal[0])
+
+
+def test_rmsnorm_against_torch_and_unit_rms():
+    x = np.random.default_rng(1).standard_normal((5, 64)) * 7.0
+    xt = torch.from_numpy(x)
+    want = xt * torch.rsqrt(xt.pow(2).mean(dim=1, keepdim=True) + 1e-6)
+    got = orc.rmsnorm(x)
+    assert np.allclose(got, want.numpy(), rtol=1e-13)
+    assert np.allclose(np.sqrt((got ** 2).mean(axis=1)), 1.0, atol=1e-6)
 
 
 @pytest.mark.parametrize("L,K", [(3, 4), (5, 3), (6, 3), (4, 6)])
