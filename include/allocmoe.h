@@ -101,6 +101,30 @@ moe_status moe_permute(const moe_shape* shape, const uint16_t* x, const int32_t*
                        int32_t* pair_pos, uint16_t* x_perm, int32_t* dev_status,
                        void* ws, size_t ws_bytes, void* stream);
 
+/* The same operation as moe_permute for callers that have no device memory of their own to lend
+ * and may not allocate any: code that runs inside a host application which handed out all GPU
+ * memory at start-up (an inference-engine plug-in, a fixed-arena embedded deployment), or a
+ * latency-critical loop in which the implicit device-wide synchronisation of cudaMalloc/cudaFree
+ * is not acceptable.  (The paper has no counterpart: it describes no permutation step.)
+ * Instead of a workspace, the per-(expert, 32-token segment) counters live in a fixed 256 KB
+ * array inside the library image, present on every GPU that loads the library until the process
+ * exits.  Inputs and outputs are passed exactly as for moe_permute and the results are identical.
+ *   Limit   N * ceil(T/32) <= 65536 (e.g. T <= 32768 at N = 64); larger shapes return
+ *           MOE_ERR_WORKSPACE and nothing is launched.
+ *   Set-up  the first call on each device looks up the array's device address (the device must
+ *           be current, as for every call); make that first call before any stream capture
+ *           begins.
+ *   Sharing all calls on a device use the one array.  Nothing in it has to start at zero (each
+ *           call writes every counter before reading it), so back-to-back calls on one stream are
+ *           fine; two calls whose kernels can overlap on the GPU (different streams) race on it
+ *           and give undefined results.
+ * The call allocates nothing and calls no allocating routine. */
+moe_status moe_permute_static(const moe_shape* shape, const uint16_t* x, const int32_t* topk_idx,
+                              const float* topk_score, const int32_t* n_sel, int64_t budget,
+                              int32_t* expert_offsets, int32_t* perm_token, float* perm_weight,
+                              int32_t* pair_pos, uint16_t* x_perm, int32_t* dev_status,
+                              void* stream);
+
 /* Routed experts ("each activated expert corresponds to one feed-forward execution",
  * Sec. 3.1).  For every listed pair p of expert e:
  *   h = silu(x_p W1_e^T) * (x_p W3_e^T)  (fp32 accumulation, h stored as bf16)

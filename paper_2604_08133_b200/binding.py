@@ -16,7 +16,7 @@ MOE_OK, MOE_ERR_ARG, MOE_ERR_BUDGET, MOE_ERR_WORKSPACE, MOE_ERR_CUDA, MOE_ERR_NO
 
 EXPORTS = ("moe_status_string", "moe_workspace_bytes", "moe_gate", "alloc_t_select", "moe_permute",
            "moe_grouped_ffn", "moe_shared_ffn", "moe_combine", "moe_layer_forward", "moe_layer_intermediates",
-           "moe_rmsnorm", "moe_profile_enable", "moe_profile_read")
+           "moe_rmsnorm", "moe_profile_enable", "moe_profile_read", "moe_permute_static")
 PROFILE_STAGES = ("gate", "select", "permute", "ffn_gemm1", "ffn_gemm2", "combine")
 
 
@@ -53,6 +53,7 @@ def lib() -> ctypes.CDLL:
             "moe_gate": [sp, vp, vp, vp, vp, vp, vp, vp],
             "alloc_t_select": [sp, vp, i64, vp, vp, vp, sz, vp],
             "moe_permute": [sp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, sz, vp],
+            "moe_permute_static": [sp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp],
             "moe_grouped_ffn": [sp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp],
             "moe_shared_ffn": [sp, vp, vp, vp, vp, vp, vp, sz, vp],
             "moe_combine": [sp, vp, vp, vp, vp, vp, vp, vp],
@@ -127,6 +128,16 @@ def moe_permute(shape, x, topk_idx, topk_score, n_sel, budget, expert_offsets, p
                                             int(budget), _p(expert_offsets), _p(perm_token), _p(perm_weight),
                                             _p(pair_pos), _p(x_perm), _p(dev_status), _p(ws), ws.numel(),
                                             _stream(stream)))
+
+
+def moe_permute_static(shape, x, topk_idx, topk_score, n_sel, budget, expert_offsets, perm_token, perm_weight, pair_pos,
+                       x_perm, dev_status, stream=None):
+    """moe_permute without a workspace argument, for callers that cannot allocate device memory:
+    the scratch is a fixed array inside the library (N * ceil(T/32) <= 65536)."""
+    _check("moe_permute_static", lib().moe_permute_static(ctypes.byref(shape), _p(x), _p(topk_idx), _p(topk_score),
+                                                          _p(n_sel), int(budget), _p(expert_offsets), _p(perm_token),
+                                                          _p(perm_weight), _p(pair_pos), _p(x_perm), _p(dev_status),
+                                                          _stream(stream)))
 
 
 def moe_grouped_ffn(shape, x_perm, expert_offsets, budget, W13, W2, y_perm, dev_status, ws, stream=None):

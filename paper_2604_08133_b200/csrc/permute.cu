@@ -143,3 +143,63 @@ moe_status launch_moe_permute(const moe_shape* s, const uint16_t* x, const int32
   }
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
+
+// ------------------------------------------------------------------------------------------------
+// moe_permute_static: moe_permute for callers that cannot allocate device memory.
+//
+// The per-(expert, 32-token segment) counters that moe_permute keeps in the caller's workspace
+// live here in a fixed array inside the library image instead.  Each GPU that loads the library
+// carries these 256 KB until the process exits.
+#include <mutex>
+
+namespace {
+
+constexpr int kStaticSegCounts = 65536;   // N * ceil(T/32) may not exceed this (256 KB of int32)
+static __device__ __align__(256) int32_t g_static_seg_counts[kStaticSegCounts];
+
+constexpr int kMaxDevices = 64;
+int32_t* g_static_seg_ptr[kMaxDevices] = {};
+std::mutex g_static_mutex;
+
+// In host code the array's name is only a handle; the address a kernel can use has to be asked for
+// while the owning device is current.  Done once per device, on that device's first call.
+moe_status static_scratch(int32_t** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MOE_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (g_static_seg_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_seg_counts) != cudaSuccess || p == nullptr) return MOE_ERR_CUDA;
+    g_static_seg_ptr[dev] = static_cast<int32_t*>(p);
+  }
+  *out = g_static_seg_ptr[dev];
+  return MOE_OK;
+}
+
+bool is_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" moe_status moe_permute_static(const moe_shape* shape, const uint16_t* x, const int32_t* topk_idx,
+                                         const float* topk_score, const int32_t* n_sel, int64_t budget,
+                                         int32_t* expert_offsets, int32_t* perm_token, float* perm_weight,
+                                         int32_t* pair_pos, uint16_t* x_perm, int32_t* dev_status, void* stream) {
+  const moe_shape* s = shape;
+  if (s == nullptr || s->flags != 0 || s->T < 1 || s->H < 64 || s->H % 64 != 0 || s->N < 8 || s->N % 8 != 0 ||
+      s->N > kMaxExperts || s->K_orig < 1 || s->K_orig > 16 || s->K_orig > s->N || s->K_base < 0 ||
+      s->K_base > s->K_orig || (long long)s->T * s->K_orig >= (1ll << 31))
+    return MOE_ERR_ARG;
+  if (!topk_idx || !topk_score || !n_sel || !expert_offsets || !perm_token || !perm_weight || !pair_pos || !dev_status)
+    return MOE_ERR_ARG;
+  if (x_perm != nullptr && (!x || !is_aligned16(x) || !is_aligned16(x_perm))) return MOE_ERR_ARG;
+  if (budget < (int64_t)s->K_base * s->T || budget > (int64_t)s->K_orig * s->T) return MOE_ERR_BUDGET;
+  // the fixed array bounds the problem size: refuse anything larger, touch nothing
+  if ((long long)s->N * ((s->T + 31) / 32) > (long long)kStaticSegCounts) return MOE_ERR_WORKSPACE;
+  int32_t* seg_counts = nullptr;
+  const moe_status st = static_scratch(&seg_counts);
+  if (st != MOE_OK) return st;
+  // Every counter a call reads is written by its own count kernel first, so whatever an earlier
+  // call left in the array needs no clearing.
+  return launch_moe_permute(s, x, topk_idx, topk_score, n_sel, budget, expert_offsets, perm_token, perm_weight,
+                            pair_pos, x_perm, dev_status, seg_counts, (cudaStream_t)stream);
+}
