@@ -19,12 +19,6 @@ DEV void set_dev_status(int32_t* dev_status, moe_status s) {
 
 DEV uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-DEV uint64_t global_timer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
 // ------------------------------------------------------------------ mbarrier
 DEV void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
@@ -47,22 +41,26 @@ DEV bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Every wait in these kernels is bounded.  A wait that exceeds kWaitLimitNs raises the CTA's
+// Every wait in these kernels is bounded.  A wait that exceeds kWaitLimitClk raises the CTA's
 // abort flag and MOE_ERR_TIMEOUT in the caller's status word; every other wait of the CTA
 // then returns false at its next poll, the roles leave their loops and the CTA tears down
-// normally (drains its own copies, frees TMEM, returns).
-constexpr uint64_t kWaitLimitNs = 500ull * 1000ull * 1000ull;   // 0.5 s
-constexpr uint64_t kDrainLimitNs = 20ull * 1000ull * 1000ull;   // teardown waits: 20 ms
+// normally (drains its own copies, frees TMEM, returns).  Time is the SM's own cycle counter,
+// looked at only every 64th poll, so a wait that succeeds quickly never pays for it.
+constexpr long long kWaitLimitClk = 1000ll * 1000ll * 1000ll;   // about 0.5 s at 1.9 GHz
+constexpr long long kDrainLimitClk = 40ll * 1000ll * 1000ll;    // teardown waits: about 20 ms
 
 DEV bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
   if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
+  long long t0 = 0;
   uint32_t spins = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((++spins & 31u) == 0u) {
+    if ((++spins & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      const long long now = clock64();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > kWaitLimitClk) {
         *abort_flag = 1;
         set_dev_status(dev_status, MOE_ERR_TIMEOUT);
         return false;
@@ -71,11 +69,41 @@ DEV bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_f
   }
 }
 
+// The same wait for a whole warp whose lanes all need the result: lane 0 polls, with a short
+// sleep between polls, and the outcome is broadcast, so that 128 epilogue threads do not all
+// poll the same barrier word.
+DEV bool mbar_wait_bounded_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
+  int ok = 1;
+  if ((threadIdx.x & 31) == 0) {
+    if (!mbar_try_wait(bar, parity)) {
+      long long t0 = 0;
+      uint32_t spins = 0;
+      while (true) {
+        __nanosleep(40);
+        if (mbar_try_wait(bar, parity)) break;
+        if ((++spins & 63u) == 0u) {
+          if (*abort_flag) { ok = 0; break; }
+          const long long now = clock64();
+          if (t0 == 0) {
+            t0 = now;
+          } else if (now - t0 > kWaitLimitClk) {
+            *abort_flag = 1;
+            set_dev_status(dev_status, MOE_ERR_TIMEOUT);
+            ok = 0;
+            break;
+          }
+        }
+      }
+    }
+  }
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
 // Teardown wait: ignores the abort flag, has its own short limit.
 DEV bool mbar_wait_drain(uint64_t* bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
-  while (global_timer_ns() - t0 < kDrainLimitNs) {
+  const long long t0 = clock64();
+  while (clock64() - t0 < kDrainLimitClk) {
     if (mbar_try_wait(bar, parity)) return true;
   }
   return false;
@@ -98,6 +126,13 @@ DEV void tma_load_3d(void* smem_dst, const void* tmap, uint64_t* bar, int c0, in
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_u32(smem_dst)), "l"((uint64_t)tmap), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+DEV void tma_load_5d(void* smem_dst, const void* tmap, uint64_t* bar, int c0, int c1, int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"((uint64_t)tmap), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
       : "memory");
 }
 
