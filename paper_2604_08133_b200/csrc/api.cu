@@ -10,6 +10,10 @@ moe_status launch_moe_gate(const moe_shape*, const uint16_t*, const uint16_t*, c
 moe_status launch_alloc_t_select(const moe_shape*, const float*, int64_t, int32_t*, int32_t*, cudaStream_t);
 moe_status launch_moe_permute(const moe_shape*, const uint16_t*, const int32_t*, const float*, const int32_t*, int64_t,
                               int32_t*, int32_t*, float*, int32_t*, uint16_t*, int32_t*, int32_t*, cudaStream_t);
+moe_status launch_gather_rows(const moe_shape*, const uint16_t*, const int32_t*, int64_t, uint16_t*, cudaStream_t);
+bool moe_route_fits(const moe_shape*);
+moe_status launch_moe_route(const moe_shape*, const float*, const int32_t*, int64_t, int32_t*, int32_t*, int32_t*, float*,
+                            int32_t*, int32_t*, cudaStream_t);
 moe_status launch_ffn(const moe_shape*, const uint16_t*, const int32_t*, int64_t, const uint16_t*, const uint16_t*,
                       uint16_t*, uint16_t*, const uint16_t*, const uint16_t*, const uint16_t*, uint16_t*, uint16_t*,
                       int32_t*, cudaStream_t, cudaEvent_t);
@@ -194,11 +198,20 @@ moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const ui
   moe_status r = launch_moe_gate(shape, x, W_gate, gate_bias, nullptr, topk_idx, topk_score, st);
   if (r != MOE_OK) return r;
   prof_mark(1, st);
-  r = launch_alloc_t_select(shape, topk_score, budget, n_sel, dev_status, st);
-  if (r != MOE_OK) return r;
-  prof_mark(2, st);
-  r = launch_moe_permute(shape, x, topk_idx, topk_score, n_sel, budget, expert_offsets, perm_token, perm_weight,
-                         pair_pos, x_perm, dev_status, at<int32_t>(ws, L.seg_counts), st);
+  if (moe_route_fits(shape)) {
+    // selection and permutation bookkeeping in one launch, then the row gather
+    r = launch_moe_route(shape, topk_score, topk_idx, budget, n_sel, expert_offsets, perm_token, perm_weight, pair_pos,
+                         dev_status, st);
+    if (r != MOE_OK) return r;
+    prof_mark(2, st);
+    if (budget > 0) r = launch_gather_rows(shape, x, perm_token, budget, x_perm, st);
+  } else {
+    r = launch_alloc_t_select(shape, topk_score, budget, n_sel, dev_status, st);
+    if (r != MOE_OK) return r;
+    prof_mark(2, st);
+    r = launch_moe_permute(shape, x, topk_idx, topk_score, n_sel, budget, expert_offsets, perm_token, perm_weight,
+                           pair_pos, x_perm, dev_status, at<int32_t>(ws, L.seg_counts), st);
+  }
   if (r != MOE_OK) return r;
   prof_mark(3, st);
   r = launch_ffn(shape, x_perm, expert_offsets, budget, W13, W2, at<uint16_t>(ws, L.h), y_perm,

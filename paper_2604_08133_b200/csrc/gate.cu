@@ -2,13 +2,20 @@
 // and the K_orig largest scores per token sorted descending (ties: lower expert id first).
 //
 // The contraction is small (2*T*H*N flops; 1 GFLOP at T=4096, H=2048, N=64) and x is read once,
-// so the kernel is bound by streaming x from HBM and by latency.  A CTA owns 32 tokens and all N
-// experts; x and W_gate chunks of 128 along H are staged in shared memory with 16-byte cp.async
-// (3 stages) and multiplied with mma.sync m16n8k16 bf16 -> fp32 (the four warps split every
-// chunk's k-steps, their partial sums are added in a fixed order).  W_gate is stored [H,N]
-// (N contiguous, the paper's R^{H x N}), which is the "column" operand of mma.sync when read
-// with ldmatrix.trans.
+// so the kernel is bound by streaming x from HBM and, at decode sizes, by latency.  A CTA owns 32
+// tokens, all N experts and every KS-th chunk of 128 along H; the KS CTAs that share a token tile
+// form a thread-block cluster (KS = 8 for H >= 1024), so that T = 64 tokens still put 16 CTAs to
+// work and no CTA walks more than a few chunks.  Chunks of x and W_gate are staged in shared
+// memory with 16-byte cp.async (3 stages) and multiplied with mma.sync m16n8k16 bf16 -> fp32; the
+// four warps split every chunk's k-steps.  Partial logits are then added in a fixed order -- warps
+// 0..3 inside a CTA, CTAs 0..KS-1 of the cluster through distributed shared memory -- and each
+// CTA finishes softmax and Top-K for its 32/KS tokens.  W_gate is stored [H,N] (N contiguous, the
+// paper's R^{H x N}), which is the "column" operand of mma.sync when read with ldmatrix.trans.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace allocmoe {
 
@@ -38,6 +45,9 @@ __global__ void __launch_bounds__(kGateThreads)
 moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ W_gate,
                 const float* __restrict__ gate_bias, int T, int H, int N, int K_orig, int w_stride,
                 float* __restrict__ scores, int32_t* __restrict__ topk_idx, float* __restrict__ topk_score) {
+  cg::cluster_group cluster = cg::this_cluster();
+  const int KS = (int)cluster.num_blocks();        // CTAs per token tile (cluster spans blockIdx.y)
+  const int ks_rank = (int)cluster.block_rank();
   constexpr int NP = NT16 * 16;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int x_stage_bytes = kGateTM * kGateXStride * 2;
@@ -45,7 +55,8 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
   const int stage_bytes = x_stage_bytes + w_stage_bytes;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int t0 = blockIdx.x * kGateTM;
-  const int nchunks = (H + kGateKC - 1) / kGateKC;
+  const int nchunks_all = (H + kGateKC - 1) / kGateKC;
+  const int nchunks = (nchunks_all - ks_rank + KS - 1) / KS;   // this CTA's chunks: ks_rank, ks_rank + KS, ...
   const int n_vec = N / 8;   // 16-byte pieces per W_gate row
 
   auto issue = [&](int chunk) {
@@ -53,7 +64,7 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
       unsigned char* st = smem_raw + (chunk % kGateStages) * stage_bytes;
       __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(st);
       __nv_bfloat16* ws = reinterpret_cast<__nv_bfloat16*>(st + x_stage_bytes);
-      const int k0 = chunk * kGateKC;
+      const int k0 = (ks_rank + chunk * KS) * kGateKC;
       for (int i = tid; i < kGateTM * (kGateKC / 8); i += kGateThreads) {
         const int r = i / (kGateKC / 8), c = i % (kGateKC / 8);
         const int t = t0 + r, k = k0 + c * 8;
@@ -133,27 +144,36 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
     v += red[(1 * kGateTM + r) * RS + c];
     v += red[(2 * kGateTM + r) * RS + c];
     v += red[(3 * kGateTM + r) * RS + c];
-    if (c < N) {
-      if (gate_bias != nullptr) v += gate_bias[c];
-    } else {
-      v = -INFINITY;
-    }
     red[r * RS + c] = v;   // row r of warp block 0: each (r,c) is read and written by this thread only
   }
-  __syncthreads();
+  cluster.sync();   // every CTA's partial logits are in its red[0 .. 32*RS)
 
-  // Softmax and sorted Top-K_orig: each warp owns 8 tokens, lane l owns experts l, l+32, ...
+  // Softmax and sorted Top-K_orig.  This CTA finishes tokens ks_rank*32/KS .. of the tile, one warp
+  // per token at a time; lane l owns experts l, l+32, ...  The KS partial sums are added in rank
+  // order, then the bias.
   constexpr int EPL = (NP + 31) / 32;
-  for (int rr = 0; rr < kGateTM / 4; ++rr) {
-    const int r = warp * (kGateTM / 4) + rr;
+  const int rows_per = kGateTM / KS;
+  const float* rred[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) rred[k] = cluster.map_shared_rank(red, k < KS ? k : 0);
+  for (int rr = warp; rr < rows_per; rr += kGateThreads / 32) {
+    const int r = ks_rank * rows_per + rr;
     const int t = t0 + r;
-    if (t >= T) break;   // uniform across the warp
+    if (t >= T) continue;   // uniform across the warp
     float v[EPL];
     float mx = -INFINITY;
 #pragma unroll
     for (int q = 0; q < EPL; ++q) {
       const int e = lane + 32 * q;
-      v[q] = (e < NP) ? red[r * RS + e] : -INFINITY;
+      float a = -INFINITY;
+      if (e < N) {
+        a = rred[0][r * RS + e];
+#pragma unroll
+        for (int k = 1; k < 8; ++k)
+          if (k < KS) a += rred[k][r * RS + e];
+        if (gate_bias != nullptr) a += gate_bias[e];
+      }
+      v[q] = a;
       mx = fmaxf(mx, v[q]);
     }
 #pragma unroll
@@ -194,6 +214,7 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
       }
     }
   }
+  cluster.sync();   // no CTA leaves while a peer may still read its partial sums
 }
 
 }  // namespace allocmoe
@@ -220,11 +241,29 @@ static moe_status gate_launch_t(const moe_shape* s, const uint16_t* x, const uin
       return MOE_ERR_CUDA;
     attr_done = true;
   }
-  const int grid = (s->T + kGateTM - 1) / kGateTM;
-  moe_gate_kernel<NT16><<<grid, kGateThreads, smem, stream>>>(
-      reinterpret_cast<const __nv_bfloat16*>(x), reinterpret_cast<const __nv_bfloat16*>(W_gate), gate_bias, s->T, s->H,
-      s->N, s->K_orig, w_stride, scores, topk_idx, topk_score);
-  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+  // CTAs per token tile: a power of two <= 8 that leaves every CTA at least one chunk, grown until
+  // the grid has about two CTAs per SM (more only adds cluster barriers)
+  const int nchunks = (s->H + kGateKC - 1) / kGateKC;
+  const int tiles = (s->T + kGateTM - 1) / kGateTM;
+  int ks = 1;
+  while (ks * 2 <= 8 && ks * 2 <= nchunks && tiles * ks < 296) ks *= 2;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)((s->T + kGateTM - 1) / kGateTM), (unsigned)ks, 1);
+  cfg.blockDim = dim3(kGateThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1;
+  attr[0].val.clusterDim.y = (unsigned)ks;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t err = cudaLaunchKernelEx(&cfg, moe_gate_kernel<NT16>, reinterpret_cast<const __nv_bfloat16*>(x),
+                                             reinterpret_cast<const __nv_bfloat16*>(W_gate), gate_bias, (int)s->T,
+                                             (int)s->H, (int)s->N, (int)s->K_orig, w_stride, scores, topk_idx,
+                                             topk_score);
+  return err == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 moe_status launch_moe_gate(const moe_shape* s, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,

@@ -10,43 +10,20 @@
 //           (expert, segment) run; expert_offsets[e] is the base of (e, 0)
 //   place : pos = base[e][seg] + rank -> perm_token, perm_weight, pair_pos
 // and a row gather x_perm[p] = x[perm_token[p]] with 128-bit loads and stores.
-#include "common.cuh"
+#include "routing.cuh"
 
 namespace allocmoe {
 
 constexpr int kPermWarps = 8;
-constexpr int kMaxExperts = 128;
-
-DEV void build_masks(uint32_t* mask, const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ n_sel,
-                     int t, int T, int N, int K_orig, int lane, int (&e_out)[16], int& n_out) {
-  for (int e = lane; e < N; e += 32) mask[e] = 0u;
-  __syncwarp();
-  n_out = 0;
-  if (t < T) {
-    n_out = min(max(n_sel[t], 0), K_orig);
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      if (j < n_out) {
-        int e = topk_idx[(long long)t * K_orig + j];
-        e = min(max(e, 0), N - 1);   // keeps every access in bounds on corrupt input
-        e_out[j] = e;
-        atomicOr(&mask[e], 1u << lane);
-      }
-    }
-  }
-  __syncwarp();
-}
 
 __global__ void __launch_bounds__(kPermWarps * 32)
 permute_count_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ n_sel, int T, int N,
                      int K_orig, int nseg, int32_t* __restrict__ seg_counts) {
   __shared__ uint32_t masks[kPermWarps][kMaxExperts];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int warp = threadIdx.x >> 5;
   const int seg = blockIdx.x * kPermWarps + warp;
   if (seg >= nseg) return;
-  int e_loc[16], n;
-  build_masks(masks[warp], topk_idx, n_sel, seg * 32 + lane, T, N, K_orig, lane, e_loc, n);
-  for (int e = lane; e < N; e += 32) seg_counts[(long long)e * nseg + seg] = __popc(masks[warp][e]);
+  permute_count_warp(masks[warp], topk_idx, n_sel, seg, T, N, K_orig, nseg, seg_counts);
 }
 
 // One CTA.  In-place exclusive scan of seg_counts (N*nseg ints, expert-major).
@@ -54,23 +31,7 @@ __global__ void __launch_bounds__(1024, 1)
 permute_scan_kernel(int32_t* __restrict__ seg_counts, int N, int nseg, long long budget,
                     int32_t* __restrict__ expert_offsets, int32_t* dev_status) {
   __shared__ int scan_ws[33];
-  const long long M = (long long)N * nseg;
-  const int per = (int)((M + blockDim.x - 1) / blockDim.x);
-  const long long lo = min(M, (long long)threadIdx.x * per), hi = min(M, lo + per);
-  int sum = 0;
-  for (long long i = lo; i < hi; ++i) sum += seg_counts[i];
-  int total;
-  int run = block_exclusive_scan(sum, scan_ws, &total);
-  for (long long i = lo; i < hi; ++i) {
-    const int c = seg_counts[i];
-    seg_counts[i] = run;
-    if (i % nseg == 0) expert_offsets[i / nseg] = run;
-    run += c;
-  }
-  if (threadIdx.x == 0) {
-    expert_offsets[N] = total;
-    if ((long long)total != budget) set_dev_status(dev_status, MOE_ERR_BUDGET);
-  }
+  permute_scan_block(seg_counts, N, nseg, budget, expert_offsets, dev_status, scan_ws);
 }
 
 __global__ void __launch_bounds__(kPermWarps * 32)
@@ -79,31 +40,11 @@ permute_place_kernel(const int32_t* __restrict__ topk_idx, const float* __restri
                      const int32_t* __restrict__ seg_base, long long budget, int32_t* __restrict__ perm_token,
                      float* __restrict__ perm_weight, int32_t* __restrict__ pair_pos) {
   __shared__ uint32_t masks[kPermWarps][kMaxExperts];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int warp = threadIdx.x >> 5;
   const int seg = blockIdx.x * kPermWarps + warp;
   if (seg >= nseg) return;
-  const int t = seg * 32 + lane;
-  int e_loc[16], n;
-  build_masks(masks[warp], topk_idx, n_sel, t, T, N, K_orig, lane, e_loc, n);
-  if (t >= T) return;
-  const uint32_t lower = (1u << lane) - 1u;
-#pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    if (j < K_orig) {
-      int pos = -1;
-      if (j < n) {
-        const int e = e_loc[j];
-        pos = seg_base[(long long)e * nseg + seg] + __popc(masks[warp][e] & lower);
-        if (pos >= 0 && pos < budget) {   // always true when sum n_sel == budget
-          perm_token[pos] = t;
-          perm_weight[pos] = topk_score[(long long)t * K_orig + j];
-        } else {
-          pos = -1;
-        }
-      }
-      pair_pos[(long long)t * K_orig + j] = pos;
-    }
-  }
+  permute_place_warp(masks[warp], topk_idx, topk_score, n_sel, seg, T, N, K_orig, nseg, seg_base, budget, perm_token,
+                     perm_weight, pair_pos);
 }
 
 // x_perm[p, :] = x[perm_token[p], :]; one CTA per row, 16 bytes per thread per step.
@@ -123,6 +64,15 @@ gather_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ perm
 
 using namespace allocmoe;
 
+moe_status launch_gather_rows(const moe_shape* s, const uint16_t* x, const int32_t* perm_token, int64_t budget,
+                              uint16_t* x_perm, cudaStream_t stream) {
+  const int row_vec = s->H / 8;
+  const long long g = budget < (1ll << 20) ? budget : (1ll << 20);
+  gather_rows_kernel<<<(unsigned)g, 256, 0, stream>>>(reinterpret_cast<const uint4*>(x), perm_token, s->T, row_vec,
+                                                      budget, reinterpret_cast<uint4*>(x_perm));
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
 size_t permute_ws_ints(const moe_shape* s) { return (size_t)s->N * ((s->T + 31) / 32); }
 
 moe_status launch_moe_permute(const moe_shape* s, const uint16_t* x, const int32_t* topk_idx, const float* topk_score,
@@ -135,12 +85,7 @@ moe_status launch_moe_permute(const moe_shape* s, const uint16_t* x, const int32
   permute_scan_kernel<<<1, 1024, 0, stream>>>(seg_counts, s->N, nseg, budget, expert_offsets, dev_status);
   permute_place_kernel<<<grid, kPermWarps * 32, 0, stream>>>(topk_idx, topk_score, n_sel, s->T, s->N, s->K_orig, nseg,
                                                              seg_counts, budget, perm_token, perm_weight, pair_pos);
-  if (x_perm != nullptr && budget > 0) {
-    const int row_vec = s->H / 8;
-    const long long g = budget < (1ll << 20) ? budget : (1ll << 20);
-    gather_rows_kernel<<<(unsigned)g, 256, 0, stream>>>(reinterpret_cast<const uint4*>(x), perm_token, s->T, row_vec,
-                                                        budget, reinterpret_cast<uint4*>(x_perm));
-  }
+  if (x_perm != nullptr && budget > 0) return launch_gather_rows(s, x, perm_token, budget, x_perm, stream);
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
