@@ -24,6 +24,7 @@ combine_kernel(const uint4* __restrict__ y_perm, const int32_t* __restrict__ pai
   __shared__ float s_w[16];
   __shared__ int s_n;
   const int t = blockIdx.x;
+  pdl_prologue_done();
   if (threadIdx.x < 16) {
     const int j = threadIdx.x;
     const int n = min(max(n_sel[t], 0), K_orig);
@@ -64,6 +65,7 @@ rmsnorm_kernel(const uint4* __restrict__ x, int row_vec, int H, uint4* __restric
   __shared__ float warp_part[8];
   __shared__ float s_scale;
   const int t = blockIdx.x;
+  pdl_prologue_done();
   float ss = 0.f;
   for (int c = threadIdx.x; c < row_vec; c += blockDim.x) {
     const uint4 v = __ldg(x + (long long)t * row_vec + c);
@@ -102,17 +104,19 @@ rmsnorm_kernel(const uint4* __restrict__ x, int row_vec, int H, uint4* __restric
 using namespace allocmoe;
 
 moe_status launch_rmsnorm(const moe_shape* s, const uint16_t* x, uint16_t* out, cudaStream_t stream) {
-  rmsnorm_kernel<<<s->T, 256, 0, stream>>>(reinterpret_cast<const uint4*>(x), s->H / 8, s->H,
-                                           reinterpret_cast<uint4*>(out));
-  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+  return launch_dependent(rmsnorm_kernel, dim3((unsigned)s->T), dim3(256), 0, stream, 1, reinterpret_cast<const uint4*>(x),
+                          s->H / 8, s->H, reinterpret_cast<uint4*>(out)) == cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
 }
 
 moe_status launch_moe_combine(const moe_shape* s, const uint16_t* y_perm, const int32_t* pair_pos,
                               const float* topk_score, const int32_t* n_sel, const uint16_t* y_shared,
                               const uint16_t* x_res, long long budget_rows, uint16_t* out, cudaStream_t stream) {
-  combine_kernel<<<s->T, 256, 0, stream>>>(reinterpret_cast<const uint4*>(y_perm), pair_pos, topk_score, n_sel,
-                                           reinterpret_cast<const uint4*>(y_shared),
-                                           reinterpret_cast<const uint4*>(x_res), s->K_orig, s->H / 8, budget_rows,
-                                           reinterpret_cast<uint4*>(out));
-  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+  return launch_dependent(combine_kernel, dim3((unsigned)s->T), dim3(256), 0, stream, 1,
+                          reinterpret_cast<const uint4*>(y_perm), pair_pos, topk_score, n_sel,
+                          reinterpret_cast<const uint4*>(y_shared), reinterpret_cast<const uint4*>(x_res), (int)s->K_orig,
+                          s->H / 8, budget_rows, reinterpret_cast<uint4*>(out)) == cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
 }

@@ -19,6 +19,17 @@ DEV void set_dev_status(int32_t* dev_status, moe_status s) {
 
 DEV uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// ------------------------------------------------------------------ programmatic dependent launch
+// Every kernel of the library is launched so that it may become resident while the previous
+// kernel of the stream is still running (launch_dependent below).  A kernel therefore does its
+// set-up that touches no global memory, calls pdl_prologue_done(), and only then reads or writes
+// global memory: the wait returns once every earlier kernel of the stream has completed and its
+// writes are visible.  Launched without the attribute, both instructions do nothing.
+DEV void pdl_prologue_done() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its own set-up
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ------------------------------------------------------------------ mbarrier
 DEV void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
@@ -245,3 +256,30 @@ DEV int block_exclusive_scan(int v, int* warp_sums, int* total) {
 }
 
 }  // namespace allocmoe
+
+// Host side: launch with the programmatic-stream-serialization attribute (and, when cluster_y > 1,
+// a thread-block cluster of (1, cluster_y, 1)).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                    unsigned cluster_y, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster_y > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = 1;
+    attr[n].val.clusterDim.y = cluster_y;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = (unsigned)n;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}

@@ -108,18 +108,8 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int kOutCols = kSwiGLU ? kUmmaN / 2 : kUmmaN;
 
-  // ---------------- setup: group table, barriers, TMEM
+  // ---------------- setup: barriers, TMEM (no global memory yet), then the group table
   const int n_groups = p.n_experts + (p.shared_rows > 0 ? 1 : 0);
-  for (int gi = tid; gi < n_groups; gi += kFfnThreads) {
-    if (gi < p.n_experts) {
-      const int lo = p.expert_offsets[gi], hi = p.expert_offsets[gi + 1];
-      ctl->row_start[gi] = lo;
-      ctl->row_count[gi] = max(hi - lo, 0);
-    } else {
-      ctl->row_start[gi] = 0;
-      ctl->row_count[gi] = p.shared_rows;
-    }
-  }
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tmem_full[a], 1); mbar_init(&ctl->tmem_empty[a], 4); }
@@ -130,6 +120,21 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
     prefetch_tensormap(&tmB_routed);
     prefetch_tensormap(&tmA_shared);
     prefetch_tensormap(&tmB_shared);
+  }
+  if (warp == 1) {
+    tmem_alloc(&ctl->tmem_base, kTmemCols);
+    tmem_relinquish();
+  }
+  pdl_prologue_done();   // expert_offsets and the operands come from earlier kernels of the stream
+  for (int gi = tid; gi < n_groups; gi += kFfnThreads) {
+    if (gi < p.n_experts) {
+      const int lo = p.expert_offsets[gi], hi = p.expert_offsets[gi + 1];
+      ctl->row_start[gi] = lo;
+      ctl->row_count[gi] = max(hi - lo, 0);
+    } else {
+      ctl->row_start[gi] = 0;
+      ctl->row_count[gi] = p.shared_rows;
+    }
   }
   __syncthreads();
   if (tid == 0) {
@@ -143,10 +148,6 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
     ctl->tile_start[n_groups] = acc;
     ctl->total_tiles = acc;
     ctl->n_groups = n_groups;
-  }
-  if (warp == 1) {
-    tmem_alloc(&ctl->tmem_base, kTmemCols);
-    tmem_relinquish();
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -368,8 +369,10 @@ static moe_status launch_gemm(const FfnGemmParams& p, const CUtensorMap& ar, con
       return MOE_ERR_CUDA;
     attr_done = true;
   }
-  ffn_gemm_kernel<kSwiGLU><<<num_sms(), kFfnThreads, kFfnSmemBytes, stream>>>(p, ar, br, as, bs);
-  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+  return launch_dependent(ffn_gemm_kernel<kSwiGLU>, dim3((unsigned)num_sms()), dim3(kFfnThreads), kFfnSmemBytes, stream, 1,
+                          p, ar, br, as, bs) == cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
 }
 
 // Routed and/or shared experts in one pair of launches.

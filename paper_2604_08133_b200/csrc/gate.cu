@@ -58,6 +58,7 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
   const int nchunks_all = (H + kGateKC - 1) / kGateKC;
   const int nchunks = (nchunks_all - ks_rank + KS - 1) / KS;   // this CTA's chunks: ks_rank, ks_rank + KS, ...
   const int n_vec = N / 8;   // 16-byte pieces per W_gate row
+  pdl_prologue_done();
 
   auto issue = [&](int chunk) {
     if (chunk < nchunks) {
@@ -247,22 +248,10 @@ static moe_status gate_launch_t(const moe_shape* s, const uint16_t* x, const uin
   const int tiles = (s->T + kGateTM - 1) / kGateTM;
   int ks = 1;
   while (ks * 2 <= 8 && ks * 2 <= nchunks && tiles * ks < 296) ks *= 2;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)((s->T + kGateTM - 1) / kGateTM), (unsigned)ks, 1);
-  cfg.blockDim = dim3(kGateThreads, 1, 1);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 1;
-  attr[0].val.clusterDim.y = (unsigned)ks;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  const cudaError_t err = cudaLaunchKernelEx(&cfg, moe_gate_kernel<NT16>, reinterpret_cast<const __nv_bfloat16*>(x),
-                                             reinterpret_cast<const __nv_bfloat16*>(W_gate), gate_bias, (int)s->T,
-                                             (int)s->H, (int)s->N, (int)s->K_orig, w_stride, scores, topk_idx,
-                                             topk_score);
+  const cudaError_t err = launch_dependent(
+      moe_gate_kernel<NT16>, dim3((unsigned)tiles, (unsigned)ks, 1), dim3(kGateThreads), smem, stream, (unsigned)ks,
+      reinterpret_cast<const __nv_bfloat16*>(x), reinterpret_cast<const __nv_bfloat16*>(W_gate), gate_bias, (int)s->T,
+      (int)s->H, (int)s->N, (int)s->K_orig, w_stride, scores, topk_idx, topk_score);
   return err == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 

@@ -22,6 +22,7 @@ permute_count_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __rest
   __shared__ uint32_t masks[kPermWarps][kMaxExperts];
   const int warp = threadIdx.x >> 5;
   const int seg = blockIdx.x * kPermWarps + warp;
+  pdl_prologue_done();
   if (seg >= nseg) return;
   permute_count_warp(masks[warp], topk_idx, n_sel, seg, T, N, K_orig, nseg, seg_counts);
 }
@@ -31,6 +32,7 @@ __global__ void __launch_bounds__(1024, 1)
 permute_scan_kernel(int32_t* __restrict__ seg_counts, int N, int nseg, long long budget,
                     int32_t* __restrict__ expert_offsets, int32_t* dev_status) {
   __shared__ int scan_ws[33];
+  pdl_prologue_done();
   permute_scan_block(seg_counts, N, nseg, budget, expert_offsets, dev_status, scan_ws);
 }
 
@@ -42,6 +44,7 @@ permute_place_kernel(const int32_t* __restrict__ topk_idx, const float* __restri
   __shared__ uint32_t masks[kPermWarps][kMaxExperts];
   const int warp = threadIdx.x >> 5;
   const int seg = blockIdx.x * kPermWarps + warp;
+  pdl_prologue_done();
   if (seg >= nseg) return;
   permute_place_warp(masks[warp], topk_idx, topk_score, n_sel, seg, T, N, K_orig, nseg, seg_base, budget, perm_token,
                      perm_weight, pair_pos);
@@ -51,6 +54,7 @@ permute_place_kernel(const int32_t* __restrict__ topk_idx, const float* __restri
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ perm_token, int T, int row_vec,
                    long long rows, uint4* __restrict__ x_perm) {
+  pdl_prologue_done();
   for (long long p = blockIdx.x; p < rows; p += gridDim.x) {
     int t = perm_token[p];
     t = min(max(t, 0), T - 1);
@@ -68,9 +72,10 @@ moe_status launch_gather_rows(const moe_shape* s, const uint16_t* x, const int32
                               uint16_t* x_perm, cudaStream_t stream) {
   const int row_vec = s->H / 8;
   const long long g = budget < (1ll << 20) ? budget : (1ll << 20);
-  gather_rows_kernel<<<(unsigned)g, 256, 0, stream>>>(reinterpret_cast<const uint4*>(x), perm_token, s->T, row_vec,
-                                                      budget, reinterpret_cast<uint4*>(x_perm));
-  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+  return launch_dependent(gather_rows_kernel, dim3((unsigned)g), dim3(256), 0, stream, 1, reinterpret_cast<const uint4*>(x),
+                          perm_token, (int)s->T, row_vec, (long long)budget, reinterpret_cast<uint4*>(x_perm)) == cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
 }
 
 size_t permute_ws_ints(const moe_shape* s) { return (size_t)s->N * ((s->T + 31) / 32); }
@@ -81,10 +86,15 @@ moe_status launch_moe_permute(const moe_shape* s, const uint16_t* x, const int32
                               int32_t* seg_counts, cudaStream_t stream) {
   const int nseg = (s->T + 31) / 32;
   const int grid = (nseg + kPermWarps - 1) / kPermWarps;
-  permute_count_kernel<<<grid, kPermWarps * 32, 0, stream>>>(topk_idx, n_sel, s->T, s->N, s->K_orig, nseg, seg_counts);
-  permute_scan_kernel<<<1, 1024, 0, stream>>>(seg_counts, s->N, nseg, budget, expert_offsets, dev_status);
-  permute_place_kernel<<<grid, kPermWarps * 32, 0, stream>>>(topk_idx, topk_score, n_sel, s->T, s->N, s->K_orig, nseg,
-                                                             seg_counts, budget, perm_token, perm_weight, pair_pos);
+  bool ok = launch_dependent(permute_count_kernel, dim3((unsigned)grid), dim3(kPermWarps * 32), 0, stream, 1, topk_idx, n_sel,
+                             (int)s->T, (int)s->N, (int)s->K_orig, nseg, seg_counts) == cudaSuccess;
+  ok = ok && launch_dependent(permute_scan_kernel, dim3(1), dim3(1024), 0, stream, 1, seg_counts, (int)s->N, nseg,
+                              (long long)budget, expert_offsets, dev_status) == cudaSuccess;
+  ok = ok && launch_dependent(permute_place_kernel, dim3((unsigned)grid), dim3(kPermWarps * 32), 0, stream, 1, topk_idx,
+                              topk_score, n_sel, (int)s->T, (int)s->N, (int)s->K_orig, nseg,
+                              static_cast<const int32_t*>(seg_counts), (long long)budget, perm_token, perm_weight,
+                              pair_pos) == cudaSuccess;
+  if (!ok) return MOE_ERR_CUDA;
   if (x_perm != nullptr && budget > 0) return launch_gather_rows(s, x, perm_token, budget, x_perm, stream);
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

@@ -26,6 +26,7 @@ moe_route_kernel(const float* __restrict__ topk_score, const int32_t* __restrict
   int32_t* seg_counts = reinterpret_cast<int32_t*>(smem_raw + sizeof(SelectSmem));
   const int warp = threadIdx.x >> 5;
   const int nseg = (T + 31) / 32;
+  pdl_prologue_done();
 
   alloc_t_select_block(smem_raw, topk_score, T, K_orig, K_base, budget - (long long)K_base * T, use_smem_keys, n_sel,
                        dev_status);   // ends with a block barrier: n_sel is visible, the pool is free
@@ -68,8 +69,9 @@ moe_status launch_moe_route(const moe_shape* s, const float* topk_score, const i
       return MOE_ERR_CUDA;
     attr_done = true;
   }
-  moe_route_kernel<<<1, kSelThreads, smem, stream>>>(topk_score, topk_idx, s->T, s->N, s->K_orig, s->K_base, budget,
-                                                     use_smem_keys, n_sel, expert_offsets, perm_token, perm_weight,
-                                                     pair_pos, dev_status);
-  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+  return launch_dependent(moe_route_kernel, dim3(1), dim3(kSelThreads), smem, stream, 1, topk_score, topk_idx, (int)s->T,
+                          (int)s->N, (int)s->K_orig, (int)s->K_base, (long long)budget, use_smem_keys, n_sel,
+                          expert_offsets, perm_token, perm_weight, pair_pos, dev_status) == cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
 }

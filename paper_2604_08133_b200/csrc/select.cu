@@ -18,6 +18,7 @@ __global__ void __launch_bounds__(kSelThreads, 1)
 alloc_t_select_kernel(const float* __restrict__ topk_score, int T, int K_orig, int K_base, long long R,
                       int use_smem_keys, int32_t* __restrict__ n_sel, int32_t* dev_status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  pdl_prologue_done();
   alloc_t_select_block(smem_raw, topk_score, T, K_orig, K_base, R, use_smem_keys, n_sel, dev_status);
 }
 
@@ -43,7 +44,8 @@ moe_status launch_alloc_t_select(const moe_shape* s, const float* topk_score, in
       return MOE_ERR_CUDA;
     attr_done = true;
   }
-  alloc_t_select_kernel<<<1, kSelThreads, smem, stream>>>(topk_score, s->T, s->K_orig, s->K_base, R, use_smem, n_sel,
-                                                          dev_status);
-  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+  return launch_dependent(alloc_t_select_kernel, dim3(1), dim3(kSelThreads), smem, stream, 1, topk_score, (int)s->T,
+                          (int)s->K_orig, (int)s->K_base, R, use_smem, n_sel, dev_status) == cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
 }
