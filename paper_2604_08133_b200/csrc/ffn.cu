@@ -255,8 +255,11 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
       const long long ld = tc.shared ? p.ld_out_shared : p.ld_out_routed;
       __nv_bfloat16* out_row = out + (long long)row * ld;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * kUmmaN;
+      // a warp whose 32 rows all lie past the end of the expert's run has nothing to store: at
+      // decode sizes (a few rows per expert) that is three warps of four
+      const int n_chunks = (tc.m0 + q * 32 < tc.m_end) ? kOutCols / 32 : 0;
 #pragma unroll 1
-      for (int c = 0; c < kOutCols / 32; ++c) {
+      for (int c = 0; c < n_chunks; ++c) {
         uint32_t packed[16];
         if (kSwiGLU) {
           uint32_t g[32], u[32];
@@ -266,8 +269,8 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
-            const float h0 = g0 * __uint_as_float(u[2 * i]) / (1.f + __expf(-g0));
-            const float h1 = g1 * __uint_as_float(u[2 * i + 1]) / (1.f + __expf(-g1));
+            const float h0 = __fdividef(g0 * __uint_as_float(u[2 * i]), 1.f + __expf(-g0));
+            const float h1 = __fdividef(g1 * __uint_as_float(u[2 * i + 1]), 1.f + __expf(-g1));
             packed[i] = pack_bf16x2(h0, h1);
           }
         } else {
