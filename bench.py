@@ -24,7 +24,10 @@ if ROOT not in sys.path:
 
 METRIC = "budgeted MoE-layer tokens/s"
 UNIT = "tokens/s"
-KERNELS_PER_STEP = 9   # gate, select, permute count/scan/place/gather, 2 expert GEMMs, combine
+def kernels_per_layer(T):
+    """Launches of one moe_layer_forward call: gate, routing (one fused launch up to 1024 tokens, else
+    select + permute count/scan/place), row gather, 2 expert GEMMs, combine."""
+    return 6 if T <= 1024 else 9
 
 
 def parse_args():
@@ -316,7 +319,7 @@ def run_ours(args):
                    "layers": n_layers, "parallelism": "independent batches per GPU, replicated weights, no collective",
                    "l2": "weights exceed L2 (no flush)" if (cfg.N + cfg.S) * 6 * cfg.H * cfg.I > 126e6 else
                          "L2-resident workload, no flush (latency-bound case)"},
-        "clocks": clocks, "gpu_launches": (KERNELS_PER_STEP + (1 if stack else 0)) * n_layers * steps,
+        "clocks": clocks, "gpu_launches": (kernels_per_layer(cfg.T) + (1 if stack else 0)) * n_layers * steps,
     }
 
     peaks = load_peaks()

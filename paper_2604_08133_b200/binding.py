@@ -16,7 +16,7 @@ MOE_OK, MOE_ERR_ARG, MOE_ERR_BUDGET, MOE_ERR_WORKSPACE, MOE_ERR_CUDA, MOE_ERR_NO
 
 EXPORTS = ("moe_status_string", "moe_workspace_bytes", "moe_gate", "alloc_t_select", "moe_permute",
            "moe_grouped_ffn", "moe_shared_ffn", "moe_combine", "moe_layer_forward", "moe_layer_intermediates",
-           "moe_rmsnorm", "moe_profile_enable", "moe_profile_read", "moe_permute_static")
+           "moe_rmsnorm", "moe_profile_enable", "moe_profile_read", "moe_permute_static", "moe_route")
 PROFILE_STAGES = ("gate", "select", "permute", "ffn_gemm1", "ffn_gemm2", "combine")
 
 
@@ -54,6 +54,7 @@ def lib() -> ctypes.CDLL:
             "alloc_t_select": [sp, vp, i64, vp, vp, vp, sz, vp],
             "moe_permute": [sp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, sz, vp],
             "moe_permute_static": [sp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp],
+            "moe_route": [sp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp],
             "moe_grouped_ffn": [sp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp],
             "moe_shared_ffn": [sp, vp, vp, vp, vp, vp, vp, sz, vp],
             "moe_combine": [sp, vp, vp, vp, vp, vp, vp, vp],
@@ -128,6 +129,14 @@ def moe_permute(shape, x, topk_idx, topk_score, n_sel, budget, expert_offsets, p
                                             int(budget), _p(expert_offsets), _p(perm_token), _p(perm_weight),
                                             _p(pair_pos), _p(x_perm), _p(dev_status), _p(ws), ws.numel(),
                                             _stream(stream)))
+
+
+def moe_route(shape, topk_idx, topk_score, budget, n_sel, expert_offsets, perm_token, perm_weight, pair_pos, dev_status,
+              stream=None):
+    """alloc_t_select + the list-building part of moe_permute in one launch (T <= 1024)."""
+    _check("moe_route", lib().moe_route(ctypes.byref(shape), _p(topk_idx), _p(topk_score), int(budget), _p(n_sel),
+                                        _p(expert_offsets), _p(perm_token), _p(perm_weight), _p(pair_pos),
+                                        _p(dev_status), _stream(stream)))
 
 
 def moe_permute_static(shape, x, topk_idx, topk_score, n_sel, budget, expert_offsets, perm_token, perm_weight, pair_pos,

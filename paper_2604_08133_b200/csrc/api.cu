@@ -138,6 +138,19 @@ moe_status moe_permute(const moe_shape* shape, const uint16_t* x, const int32_t*
                             pair_pos, x_perm, dev_status, at<int32_t>(ws, L.seg_counts), (cudaStream_t)stream);
 }
 
+moe_status moe_route(const moe_shape* shape, const int32_t* topk_idx, const float* topk_score, int64_t budget,
+                     int32_t* n_sel, int32_t* expert_offsets, int32_t* perm_token, float* perm_weight, int32_t* pair_pos,
+                     int32_t* dev_status, void* stream) {
+  if (!shape_ok(shape) || !topk_idx || !topk_score || !n_sel || !expert_offsets || !perm_token || !perm_weight ||
+      !pair_pos || !dev_status)
+    return MOE_ERR_ARG;
+  if (!aligned16(topk_idx) || !aligned16(topk_score) || !aligned16(n_sel)) return MOE_ERR_ARG;
+  if (!moe_route_fits(shape)) return MOE_ERR_ARG;
+  if (!budget_ok(shape, budget)) return MOE_ERR_BUDGET;
+  return launch_moe_route(shape, topk_score, topk_idx, budget, n_sel, expert_offsets, perm_token, perm_weight, pair_pos,
+                          dev_status, (cudaStream_t)stream);
+}
+
 moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_perm, const int32_t* expert_offsets,
                            int64_t budget, const uint16_t* W13, const uint16_t* W2, uint16_t* y_perm,
                            int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {

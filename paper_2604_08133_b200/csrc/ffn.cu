@@ -13,12 +13,13 @@
 // A "group" is a routed expert or, last, the shared experts (all T rows; their S sub-experts
 // are extra column blocks in GEMM-1 and extra K blocks in GEMM-2).
 //
-// CTA = 6 warps: warp 0 lane 0 issues TMA loads (A 128x64, B 256x64 bf16, 128-byte swizzle)
-// into a 4-stage ring; warp 1 lane 0 issues tcgen05.mma (M=128, N=256, K=16) into one of two
-// 256-column TMEM accumulators; warps 2-5 read the finished accumulator with tcgen05.ld, apply
+// CTA = 6 warps: warp 0 lane 0 issues TMA loads (A 128x64, B 256x64 or 128x64 bf16, 128-byte
+// swizzle) into a ring of 4 (6) stages; warp 1 lane 0 issues tcgen05.mma (M=128, N=256 or 128,
+// K=16) into one of two TMEM accumulators; warps 2-5 read the finished accumulator with tcgen05.ld, apply
 // the epilogue and store bf16 rows (row-masked at the ragged end of an expert's run) while the
 // next tile's main loop runs.  Every mbarrier wait is bounded (see common.cuh).
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -26,13 +27,20 @@ namespace allocmoe {
 
 constexpr int kBM = 128;            // rows per tile (UMMA M)
 constexpr int kBK = 64;             // K per stage: 64 bf16 = one 128-byte swizzle row
-constexpr int kUmmaN = 256;         // accumulator columns per tile
-constexpr int kStages = 4;
+constexpr int kAccCols = 256;       // TMEM columns reserved per accumulator
+constexpr int kMaxStages = 6;
 constexpr int kFfnThreads = 192;
 constexpr int kABytes = kBM * kBK * 2;        // 16 KB
-constexpr int kBBytes = kUmmaN * kBK * 2;     // 32 KB
-constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kTmemCols = 512;      // two accumulators of 256 columns
+
+// The B tile (weight rows = UMMA N) is 256 rows (4 stages of 48 KB) or 128 rows (6 stages of 32 KB).
+template <int kN>
+struct TileCfg {
+  static constexpr int kBBytes = kN * kBK * 2;             // 32 or 16 KB
+  static constexpr int kStageBytes = kABytes + kBBytes;    // 48 or 32 KB
+  static constexpr int kStages = kN == 256 ? 4 : 6;
+  static constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes;
+};
 constexpr int kMaxGroups = 130;     // up to 128 routed experts + the shared group
 
 struct FfnGemmParams {
@@ -50,8 +58,8 @@ struct FfnGemmParams {
 };
 
 struct FfnSmemCtl {
-  uint64_t full[kStages];
-  uint64_t empty[kStages];
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
   uint64_t drain;
@@ -69,15 +77,15 @@ struct TileCoord {
   bool shared;
 };
 
-// kSwiGLU: true = GEMM-1 (B tile = 128 W1 rows + 128 W3 rows, 128 output columns),
-//          false = GEMM-2 (B tile = 256 W2 rows, 256 output columns).
-template <bool kSwiGLU>
+// kSwiGLU: true = GEMM-1 (B tile = kN/2 W1 rows + kN/2 W3 rows, kN/2 output columns),
+//          false = GEMM-2 (B tile = kN W2 rows, kN output columns).
+template <bool kSwiGLU, int kN>
 struct TileWalker {
   const FfnSmemCtl* c;
   int nb_routed, nb_shared;
   int g;
   DEV TileWalker(const FfnSmemCtl* ctl, const FfnGemmParams& p) : c(ctl), g(0) {
-    constexpr int cols = kSwiGLU ? kUmmaN / 2 : kUmmaN;
+    constexpr int cols = kSwiGLU ? kN / 2 : kN;
     nb_routed = (p.n_per_sub + cols - 1) / cols;
     nb_shared = kSwiGLU ? nb_routed * p.shared_sub : nb_routed;
   }
@@ -96,7 +104,7 @@ struct TileWalker {
   }
 };
 
-template <bool kSwiGLU>
+template <bool kSwiGLU, int kN>
 __global__ void __launch_bounds__(kFfnThreads, 1)
 ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_routed,
                 const __grid_constant__ CUtensorMap tmB_routed, const __grid_constant__ CUtensorMap tmA_shared,
@@ -104,9 +112,10 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   extern __shared__ unsigned char smem_dyn[];
   // tiles need 1024-byte alignment for the 128-byte swizzle
   unsigned char* tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
-  FfnSmemCtl* ctl = reinterpret_cast<FfnSmemCtl*>(tiles + kStages * kStageBytes);
+  FfnSmemCtl* ctl = reinterpret_cast<FfnSmemCtl*>(tiles + TileCfg<kN>::kSmemBytes);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  constexpr int kOutCols = kSwiGLU ? kUmmaN / 2 : kUmmaN;
+  constexpr int kStages = TileCfg<kN>::kStages, kStageBytes = TileCfg<kN>::kStageBytes, kBBytes = TileCfg<kN>::kBBytes;
+  constexpr int kOutCols = kSwiGLU ? kN / 2 : kN;
 
   // ---------------- setup: barriers, TMEM (no global memory yet), then the group table
   const int n_groups = p.n_experts + (p.shared_rows > 0 ? 1 : 0);
@@ -138,7 +147,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   }
   __syncthreads();
   if (tid == 0) {
-    TileWalker<kSwiGLU> w(ctl, p);
+    TileWalker<kSwiGLU, kN> w(ctl, p);
     int acc = 0;
     for (int gi = 0; gi < n_groups; ++gi) {
       ctl->tile_start[gi] = acc;
@@ -161,7 +170,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   if (warp == 0) {
     // ======================= TMA producer =======================
     if (lane == 0) {
-      TileWalker<kSwiGLU> w(ctl, p);
+      TileWalker<kSwiGLU, kN> w(ctl, p);
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
@@ -201,8 +210,8 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   } else if (warp == 1) {
     // ======================= MMA issuer =======================
     if (lane == 0) {
-      TileWalker<kSwiGLU> w(ctl, p);
-      constexpr uint32_t idesc = umma_idesc_bf16(kBM, kUmmaN);
+      TileWalker<kSwiGLU, kN> w(ctl, p);
+      constexpr uint32_t idesc = umma_idesc_bf16(kBM, kN);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
@@ -211,7 +220,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
         const uint32_t a = tcount & 1u, aph = (tcount >> 1) & 1u;
         if (!(ok = mbar_wait_bounded(&ctl->tmem_empty[a], aph ^ 1u, abort_flag, p.dev_status))) break;
         tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + a * kUmmaN;
+        const uint32_t d_tmem = tmem_base + a * kAccCols;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
@@ -232,7 +241,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
     }
   } else {
     // ======================= epilogue (warps 2..5) =======================
-    TileWalker<kSwiGLU> w(ctl, p);
+    TileWalker<kSwiGLU, kN> w(ctl, p);
     const int q = warp & 3;                  // TMEM lane quarter this warp may read
     uint32_t tcount = 0;
     bool ok = true;
@@ -254,7 +263,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
       __nv_bfloat16* out = tc.shared ? p.out_shared : p.out_routed;
       const long long ld = tc.shared ? p.ld_out_shared : p.ld_out_routed;
       __nv_bfloat16* out_row = out + (long long)row * ld;
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * kUmmaN;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * kAccCols;
       // a warp whose 32 rows all lie past the end of the expert's run has nothing to store: at
       // decode sizes (a few rows per expert) that is three warps of four
       const int n_chunks = (tc.m0 + q * 32 < tc.m_end) ? kOutCols / 32 : 0;
@@ -264,7 +273,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
         if (kSwiGLU) {
           uint32_t g[32], u[32];
           tmem_ld_32x32(taddr + c * 32, g);
-          tmem_ld_32x32(taddr + kUmmaN / 2 + c * 32, u);
+          tmem_ld_32x32(taddr + kN / 2 + c * 32, u);
           tmem_ld_wait();
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
@@ -360,22 +369,36 @@ static int num_sms() {
   return g_num_sms;
 }
 
-constexpr size_t kFfnSmemBytes = (size_t)kStages * kStageBytes + sizeof(FfnSmemCtl) + 1024;
 
-template <bool kSwiGLU>
+template <bool kSwiGLU, int kN>
 static moe_status launch_gemm(const FfnGemmParams& p, const CUtensorMap& ar, const CUtensorMap& br,
                               const CUtensorMap& as, const CUtensorMap& bs, cudaStream_t stream) {
+  constexpr size_t smem = TileCfg<kN>::kSmemBytes + sizeof(FfnSmemCtl) + 1024;
+  static_assert(smem <= 232448, "ring + control block exceed the 227 KB a CTA may use");
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(ffn_gemm_kernel<kSwiGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kFfnSmemBytes) != cudaSuccess)
+    if (cudaFuncSetAttribute(ffn_gemm_kernel<kSwiGLU, kN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
       return MOE_ERR_CUDA;
     attr_done = true;
   }
-  return launch_dependent(ffn_gemm_kernel<kSwiGLU>, dim3((unsigned)num_sms()), dim3(kFfnThreads), kFfnSmemBytes, stream, 1,
-                          p, ar, br, as, bs) == cudaSuccess
+  return launch_dependent(ffn_gemm_kernel<kSwiGLU, kN>, dim3((unsigned)num_sms()), dim3(kFfnThreads), smem, stream, 1, p,
+                          ar, br, as, bs) == cudaSuccess
              ? MOE_OK
              : MOE_ERR_CUDA;
+}
+
+// Weight rows per tile.  256 everywhere: the 128-row variant (twice as many, half as long tiles, 6
+// stages) was measured slower on every workload -- each tile re-reads its 16 KB token stage from
+// L2 twice as often -- and is kept only behind the knob.
+static int pick_tile_n(const moe_shape*, int64_t, bool) {
+  static int forced = -1;
+  if (forced < 0) {
+    forced = 0;
+    const char* e = getenv("ALLOCMOE_TILE_N");   // tuning knob: 128 or 256
+    if (e != nullptr && (atoi(e) == 128 || atoi(e) == 256)) forced = atoi(e);
+  }
+  return forced ? forced : 256;
 }
 
 // Routed and/or shared experts in one pair of launches.
@@ -389,6 +412,8 @@ moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t*
   if (!routed && !shared) return MOE_OK;
   const uint64_t H = s->H, I = s->I;
   CUtensorMap a1r, b1r, a1s, b1s, a2r, b2r, a2s, b2s;
+  const int tile_n = pick_tile_n(s, routed ? budget : 0, shared);
+  const uint32_t kUmmaN = (uint32_t)tile_n;
   bool ok = true;
   if (routed) {
     ok &= make_tmap(&a1r, x_perm, H, (uint64_t)budget, 0, H, 0, kBM);
@@ -421,7 +446,8 @@ moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t*
   p.out_shared = reinterpret_cast<__nv_bfloat16*>(h_sh);
   p.ld_out_routed = s->I;
   p.ld_out_shared = (long long)s->S * s->I;
-  moe_status st = launch_gemm<true>(p, a1r, b1r, a1s, b1s, stream);
+  moe_status st = tile_n == 128 ? launch_gemm<true, 128>(p, a1r, b1r, a1s, b1s, stream)
+                                : launch_gemm<true, 256>(p, a1r, b1r, a1s, b1s, stream);
   if (st != MOE_OK) return st;
   if (between != nullptr) cudaEventRecord(between, stream);
   // GEMM-2
@@ -432,5 +458,6 @@ moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t*
   p.out_shared = reinterpret_cast<__nv_bfloat16*>(y_shared);
   p.ld_out_routed = s->H;
   p.ld_out_shared = s->H;
-  return launch_gemm<false>(p, a2r, b2r, a2s, b2s, stream);
+  return tile_n == 128 ? launch_gemm<false, 128>(p, a2r, b2r, a2s, b2s, stream)
+                       : launch_gemm<false, 256>(p, a2r, b2r, a2s, b2s, stream);
 }

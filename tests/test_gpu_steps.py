@@ -108,6 +108,47 @@ def test_moe_permute_bit_exact(T, N, K, kb, mult):
     assert torch.equal(xp.cpu(), x.cpu()[torch.from_numpy(want["perm_token"]).long()])
 
 
+@pytest.mark.parametrize("T,N,K,kb,mult,ties", [(1, 8, 2, 1, 1.0, False), (64, 8, 2, 0, 1.0, False),
+                                                 (64, 64, 6, 1, 3.0, False), (333, 16, 4, 0, 1.3, True),
+                                                 (1000, 64, 6, 1, 2.5, True), (1024, 128, 8, 2, 5.0, False),
+                                                 (1024, 64, 6, 1, 6.0, False), (1024, 64, 6, 1, 1.0, False)])
+def test_moe_route_fused_bit_exact(T, N, K, kb, mult, ties):
+    """The one-launch routing step gives what the oracle's selection and permutation give, ties included."""
+    g = torch.Generator().manual_seed(T * 17 + N)
+    logits = torch.randn(T, N, generator=g, dtype=torch.float64)
+    if ties:                                   # quantised logits: many equal scores inside and across tokens
+        logits = torch.round(logits * 2) / 2
+    p = orc.softmax_scores(logits.numpy())
+    idx, sc = orc.topk_sorted(p, K)
+    budget = max(kb * T, min(K * T, int(mult * T)))
+    n_ref = orc.n_sel_from_mask(orc.alloc_t_select_threshold(sc, kb, budget))
+    want = orc.permute(idx, sc, n_ref, N)
+    shape = B.make_shape(T, 64, N, 64, 0, K, kb)
+    n_sel = torch.full((T,), -3, dtype=torch.int32, device="cuda")
+    off = torch.empty(N + 1, dtype=torch.int32, device="cuda")
+    tok = torch.empty(max(budget, 1), dtype=torch.int32, device="cuda")
+    wgt = torch.empty(max(budget, 1), dtype=torch.float32, device="cuda")
+    pos = torch.empty(T, K, dtype=torch.int32, device="cuda")
+    st = _status()
+    for _ in range(2):                         # twice: nothing may depend on what the first call left behind
+        B.moe_route(shape, torch.from_numpy(idx).cuda(), torch.from_numpy(sc).cuda(), budget, n_sel, off, tok, wgt, pos, st)
+        torch.cuda.synchronize()
+        assert st.item() == 0
+        assert np.array_equal(n_sel.cpu().numpy(), n_ref)
+        assert np.array_equal(off.cpu().numpy(), want["expert_offsets"])
+        assert np.array_equal(tok.cpu().numpy()[:budget], want["perm_token"])
+        assert np.array_equal(wgt.cpu().numpy()[:budget], want["perm_weight"])
+        assert np.array_equal(pos.cpu().numpy(), want["pair_pos"])
+
+
+def test_moe_route_refuses_large_batches():
+    shape = B.make_shape(2048, 64, 64, 64, 0, 6, 1)
+    z = torch.zeros(2048 * 6, dtype=torch.int32, device="cuda")
+    with pytest.raises(B.MoeError) as ei:
+        B.moe_route(shape, z, z.float(), 4096, z, z, z, z.float(), z, _status())
+    assert ei.value.status == B.MOE_ERR_ARG
+
+
 def test_moe_permute_flags_a_count_mismatch():
     T, N, K = 64, 8, 2
     shape = B.make_shape(T, 64, N, 64, 0, K, 0)
