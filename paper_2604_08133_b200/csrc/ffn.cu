@@ -79,7 +79,7 @@ struct TileCoord {
 
 // kSwiGLU: true = GEMM-1 (B tile = kN/2 W1 rows + kN/2 W3 rows, kN/2 output columns),
 //          false = GEMM-2 (B tile = kN W2 rows, kN output columns).
-template <bool kSwiGLU, int kN>
+template <bool kSwiGLU, int kN, int kTileM>
 struct TileWalker {
   const FfnSmemCtl* c;
   int nb_routed, nb_shared;
@@ -95,10 +95,10 @@ struct TileWalker {
     tc.group = g;
     tc.shared = (g >= p.n_experts);
     const int local = tile - c->tile_start[g];
-    const int mblocks = (c->row_count[g] + kBM - 1) / kBM;
+    const int mblocks = (c->row_count[g] + kTileM - 1) / kTileM;
     tc.nb = local / mblocks;
     const int mb = local % mblocks;
-    tc.m0 = c->row_start[g] + mb * kBM;
+    tc.m0 = c->row_start[g] + mb * kTileM;
     tc.m_end = c->row_start[g] + c->row_count[g];
     return tc;
   }
@@ -147,7 +147,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   }
   __syncthreads();
   if (tid == 0) {
-    TileWalker<kSwiGLU, kN> w(ctl, p);
+    TileWalker<kSwiGLU, kN, kBM> w(ctl, p);
     int acc = 0;
     for (int gi = 0; gi < n_groups; ++gi) {
       ctl->tile_start[gi] = acc;
@@ -170,7 +170,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   if (warp == 0) {
     // ======================= TMA producer =======================
     if (lane == 0) {
-      TileWalker<kSwiGLU, kN> w(ctl, p);
+      TileWalker<kSwiGLU, kN, kBM> w(ctl, p);
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
@@ -210,7 +210,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   } else if (warp == 1) {
     // ======================= MMA issuer =======================
     if (lane == 0) {
-      TileWalker<kSwiGLU, kN> w(ctl, p);
+      TileWalker<kSwiGLU, kN, kBM> w(ctl, p);
       constexpr uint32_t idesc = umma_idesc_bf16(kBM, kN);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
@@ -241,7 +241,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
     }
   } else {
     // ======================= epilogue (warps 2..5) =======================
-    TileWalker<kSwiGLU, kN> w(ctl, p);
+    TileWalker<kSwiGLU, kN, kBM> w(ctl, p);
     const int q = warp & 3;                  // TMEM lane quarter this warp may read
     uint32_t tcount = 0;
     bool ok = true;
@@ -320,6 +320,246 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// The same GEMM on CTA pairs (cta_group::2).  A cluster of two CTAs on the two SMs of a TPC works on
+// a tile of 256 rows x 256 weight rows: each CTA loads its own 128 rows of A and HALF of the B tile
+// (for GEMM-1 the leader takes the 128 W1 rows, its peer the 128 W3 rows), the leader's MMA thread
+// issues tcgen05.mma with M = 256 and both tensor cores read the two halves of B from both shared
+// memories.  Per 128x256x64 block of MACs an SM now moves 32 KB from L2 instead of 48 KB and reads
+// 8 KB instead of 12 KB of operands per MMA from shared memory -- the two paths that bound the
+// one-CTA kernel on compute-heavy shapes -- and the ring holds 6 stages.
+//
+// Barriers: `full` lives in the leader and counts two arrivals (each CTA's producer announces its
+// own 32 KB); `empty` and `tmem_full` exist in both CTAs and are signalled by multicast commits;
+// `tmem_empty` lives in the leader and counts the 8 epilogue warps of the pair.  No load uses
+// cluster multicast.
+constexpr int kPairStages = 6;
+constexpr int kPairStageBytes = 2 * kABytes;          // 16 KB of A + 16 KB of B per CTA
+constexpr int kPairM = 2 * kBM;
+
+template <bool kSwiGLU>
+__global__ void __launch_bounds__(kFfnThreads, 1)
+ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_routed,
+                     const __grid_constant__ CUtensorMap tmB_routed, const __grid_constant__ CUtensorMap tmA_shared,
+                     const __grid_constant__ CUtensorMap tmB_shared) {
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  FfnSmemCtl* ctl = reinterpret_cast<FfnSmemCtl*>(tiles + kPairStages * kPairStageBytes);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int kN = 256;
+  constexpr int kOutCols = kSwiGLU ? kN / 2 : kN;
+  const uint32_t rank = cluster_cta_rank();          // 0 = leader
+  const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  // ---------------- setup: barriers, TMEM (no global memory yet), then the group table
+  const int n_groups = p.n_experts + (p.shared_rows > 0 ? 1 : 0);
+  if (tid == 0) {
+    for (int s = 0; s < kPairStages; ++s) { mbar_init(&ctl->full[s], 2); mbar_init(&ctl->empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tmem_full[a], 1); mbar_init(&ctl->tmem_empty[a], 8); }
+    mbar_init(&ctl->drain, 1);
+    ctl->abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tensormap(&tmA_routed);
+    prefetch_tensormap(&tmB_routed);
+    prefetch_tensormap(&tmA_shared);
+    prefetch_tensormap(&tmB_shared);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(&ctl->tmem_base, kTmemCols);
+    tmem_relinquish_pair();
+  }
+  pdl_prologue_done();
+  for (int gi = tid; gi < n_groups; gi += kFfnThreads) {
+    if (gi < p.n_experts) {
+      const int lo = p.expert_offsets[gi], hi = p.expert_offsets[gi + 1];
+      ctl->row_start[gi] = lo;
+      ctl->row_count[gi] = max(hi - lo, 0);
+    } else {
+      ctl->row_start[gi] = 0;
+      ctl->row_count[gi] = p.shared_rows;
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    TileWalker<kSwiGLU, kN, kPairM> w(ctl, p);
+    int acc = 0;
+    for (int gi = 0; gi < n_groups; ++gi) {
+      ctl->tile_start[gi] = acc;
+      const int mblocks = (ctl->row_count[gi] + kPairM - 1) / kPairM;
+      acc += mblocks * (gi < p.n_experts ? w.nb_routed : w.nb_shared);
+    }
+    ctl->tile_start[n_groups] = acc;
+    ctl->total_tiles = acc;
+    ctl->n_groups = n_groups;
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();          // both CTAs' barriers are initialised before either signals the other
+  tc_fence_after_sync();
+  const uint32_t tmem_base = ctl->tmem_base;
+  const int total_tiles = ctl->total_tiles;
+  const int kb_routed = p.k_per_sub / kBK;
+  const int kb_shared = kSwiGLU ? kb_routed : kb_routed * p.shared_sub;
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  if (warp == 0) {
+    // ======================= TMA producer (both CTAs) =======================
+    if (lane == 0) {
+      TileWalker<kSwiGLU, kN, kPairM> w(ctl, p);
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs) {
+        const TileCoord tc = w.at(tile, p);
+        const CUtensorMap* tmA = tc.shared ? &tmA_shared : &tmA_routed;
+        const CUtensorMap* tmB = tc.shared ? &tmB_shared : &tmB_routed;
+        const int nkb = tc.shared ? kb_shared : kb_routed;
+        int e_n = tc.group, n_row = tc.nb * kOutCols;
+        if (tc.shared) {
+          if (kSwiGLU) { e_n = tc.nb / w.nb_routed; n_row = (tc.nb % w.nb_routed) * kOutCols; }
+          else { e_n = 0; }
+        }
+        // this CTA's half of the B tile: GEMM-1 W1 rows (leader) or W3 rows (peer); GEMM-2 rows +128*rank
+        const int b_row = kSwiGLU ? (rank == 0 ? n_row : p.up_row_offset + n_row) : n_row + (int)rank * (kN / 2);
+        const int a_row = tc.m0 + (int)rank * kBM;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % kPairStages;
+          const uint32_t ph = (it / kPairStages) & 1u;
+          if (!(ok = mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status))) break;
+          unsigned char* sa = tiles + s * kPairStageBytes;
+          unsigned char* sb = sa + kABytes;
+          const uint32_t bar = cluster_addr_of(&ctl->full[s], 0);
+          mbar_expect_tx_cluster(bar, kPairStageBytes);
+          tma_load_2d_pair(sa, tmA, bar, kb * kBK, a_row);
+          int e_k = e_n, k_col = kb * kBK;
+          if (tc.shared && !kSwiGLU) { e_k = kb / kb_routed; k_col = (kb % kb_routed) * kBK; }
+          tma_load_3d_pair(sb, tmB, bar, k_col, b_row, e_k);
+        }
+      }
+      // drain: the last loads have landed once the leader's barriers of the last stages completed;
+      // the peer learns it through the multicast `empty` that follows.  Wait for what was issued.
+      const uint32_t issued = it;
+      if (rank == 0) {
+        for (uint32_t q = (issued > (uint32_t)kPairStages ? issued - kPairStages : 0u); q < issued; ++q)
+          mbar_wait_drain(&ctl->full[q % kPairStages], (q / kPairStages) & 1u);
+      } else {
+        for (uint32_t q = (issued > (uint32_t)kPairStages ? issued - kPairStages : 0u); q < issued; ++q)
+          mbar_wait_drain(&ctl->empty[q % kPairStages], (q / kPairStages) & 1u);
+      }
+    }
+  } else if (warp == 1) {
+    // ======================= MMA issuer (leader only) =======================
+    if (lane == 0 && rank == 0) {
+      TileWalker<kSwiGLU, kN, kPairM> w(ctl, p);
+      constexpr uint32_t idesc = umma_idesc_bf16(kPairM, kN);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs, ++tcount) {
+        const TileCoord tc = w.at(tile, p);
+        const int nkb = tc.shared ? kb_shared : kb_routed;
+        const uint32_t a = tcount & 1u, aph = (tcount >> 1) & 1u;
+        if (!(ok = mbar_wait_bounded(&ctl->tmem_empty[a], aph ^ 1u, abort_flag, p.dev_status))) break;
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + a * kAccCols;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % kPairStages;
+          const uint32_t ph = (it / kPairStages) & 1u;
+          if (!(ok = mbar_wait_bounded(&ctl->full[s], ph, abort_flag, p.dev_status))) break;
+          tc_fence_after_sync();
+          const uint32_t sa = smem_u32(tiles + s * kPairStageBytes);
+          const uint64_t da = umma_desc_sw128(sa), db = umma_desc_sw128(sa + kABytes);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k)
+            umma_bf16_pair(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+          umma_commit_pair(&ctl->empty[s], 3);      // frees the stage in both CTAs
+        }
+        if (ok) umma_commit_pair(&ctl->tmem_full[a], 3);
+      }
+      // drain: all MMAs complete before TMEM is freed
+      umma_commit_pair(&ctl->drain, 1);
+      mbar_wait_drain(&ctl->drain, 0u);
+    }
+  } else {
+    // ======================= epilogue (warps 2..5 of both CTAs) =======================
+    TileWalker<kSwiGLU, kN, kPairM> w(ctl, p);
+    const int q = warp & 3;
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs, ++tcount) {
+      const TileCoord tc = w.at(tile, p);
+      const uint32_t a = tcount & 1u, aph = (tcount >> 1) & 1u;
+      if (!(ok = mbar_wait_bounded_warp(&ctl->tmem_full[a], aph, abort_flag, p.dev_status))) break;
+      tc_fence_after_sync();
+      const int row0 = tc.m0 + (int)rank * kBM + q * 32;
+      const int row = row0 + lane;
+      const bool row_ok = row < tc.m_end;
+      const int n_total = tc.shared ? (kSwiGLU ? p.n_per_sub * p.shared_sub : p.n_per_sub) : p.n_per_sub;
+      int col0 = tc.nb * kOutCols;
+      int col_limit = n_total;
+      if (kSwiGLU && tc.shared) {
+        const int s = tc.nb / w.nb_routed;
+        col0 = s * p.n_per_sub + (tc.nb % w.nb_routed) * kOutCols;
+        col_limit = (s + 1) * p.n_per_sub;
+      }
+      __nv_bfloat16* out = tc.shared ? p.out_shared : p.out_routed;
+      const long long ld = tc.shared ? p.ld_out_shared : p.ld_out_routed;
+      __nv_bfloat16* out_row = out + (long long)row * ld;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * kAccCols;
+      const int n_chunks = (row0 < tc.m_end) ? kOutCols / 32 : 0;
+#pragma unroll 1
+      for (int c = 0; c < n_chunks; ++c) {
+        uint32_t packed[16];
+        if (kSwiGLU) {
+          uint32_t g[32], u[32];
+          tmem_ld_32x32(taddr + c * 32, g);
+          tmem_ld_32x32(taddr + kN / 2 + c * 32, u);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+            const float h0 = __fdividef(g0 * __uint_as_float(u[2 * i]), 1.f + __expf(-g0));
+            const float h1 = __fdividef(g1 * __uint_as_float(u[2 * i + 1]), 1.f + __expf(-g1));
+            packed[i] = pack_bf16x2(h0, h1);
+          }
+        } else {
+          uint32_t v[32];
+          tmem_ld_32x32(taddr + c * 32, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) packed[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+        }
+        const int col = col0 + c * 32;
+        if (row_ok) {
+          if (col + 32 <= col_limit) {
+            uint4* dst = reinterpret_cast<uint4*>(out_row + col);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+          } else {
+            for (int i = 0; i < 32; ++i)
+              if (col + i < col_limit) {
+                const uint32_t w2 = packed[i >> 1];
+                reinterpret_cast<uint16_t*>(out_row)[col + i] = (uint16_t)((i & 1) ? (w2 >> 16) : (w2 & 0xFFFFu));
+              }
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(cluster_addr_of(&ctl->tmem_empty[a], 0));
+    }
+  }
+
+  // ---------------- teardown: neither CTA leaves (or frees TMEM) while its peer may still touch it
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
+  }
+}
+
 }  // namespace allocmoe
 
 using namespace allocmoe;
@@ -388,6 +628,41 @@ static moe_status launch_gemm(const FfnGemmParams& p, const CUtensorMap& ar, con
              : MOE_ERR_CUDA;
 }
 
+template <bool kSwiGLU>
+static moe_status launch_gemm_pair(const FfnGemmParams& p, const CUtensorMap& ar, const CUtensorMap& br,
+                                   const CUtensorMap& as, const CUtensorMap& bs, cudaStream_t stream) {
+  constexpr size_t smem = (size_t)kPairStages * kPairStageBytes + sizeof(FfnSmemCtl) + 1024;
+  static_assert(smem <= 232448, "ring + control block exceed the 227 KB a CTA may use");
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(ffn_gemm_pair_kernel<kSwiGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
+      return MOE_ERR_CUDA;
+    attr_done = true;
+  }
+  const unsigned grid = (unsigned)(num_sms() & ~1);
+  return launch_dependent_cluster(ffn_gemm_pair_kernel<kSwiGLU>, dim3(grid), dim3(kFfnThreads), smem, stream,
+                                  dim3(2, 1, 1), p, ar, br, as, bs) == cudaSuccess
+             ? MOE_OK
+             : MOE_ERR_CUDA;
+}
+
+// CTA pairs or single CTAs.  Measured on B200: pairs win (7 % of the layer) where the routed experts
+// receive between 128 and 256 rows on average -- one 256-row pair tile then covers an expert that
+// needs two single-CTA tiles, the second mostly padding; they lose at decode sizes (the HBM-bound
+// stream runs with half as many weight bytes per stage) and on very large experts under the
+// power cap.  ALLOCMOE_PAIR = 0 / 1 forces the choice.
+static bool use_pairs(const moe_shape* s, int64_t routed_rows) {
+  static int forced = -2;
+  if (forced == -2) {
+    forced = -1;
+    const char* e = getenv("ALLOCMOE_PAIR");
+    if (e != nullptr) forced = atoi(e) != 0 ? 1 : 0;
+  }
+  if (forced >= 0) return forced == 1;
+  return routed_rows > 128ll * s->N && routed_rows <= 256ll * s->N;
+}
+
 // Weight rows per tile.  256 everywhere: the 128-row variant (twice as many, half as long tiles, 6
 // stages) was measured slower on every workload -- each tile re-reads its 16 KB token stage from
 // L2 twice as often -- and is kept only behind the knob.
@@ -412,21 +687,23 @@ moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t*
   if (!routed && !shared) return MOE_OK;
   const uint64_t H = s->H, I = s->I;
   CUtensorMap a1r, b1r, a1s, b1s, a2r, b2r, a2s, b2s;
-  const int tile_n = pick_tile_n(s, routed ? budget : 0, shared);
+  const bool pairs = use_pairs(s, routed ? budget : 0);
+  const int tile_n = pairs ? 256 : pick_tile_n(s, routed ? budget : 0, shared);
   const uint32_t kUmmaN = (uint32_t)tile_n;
+  const uint32_t b2_box = pairs ? kUmmaN / 2 : kUmmaN;   // a pair's CTA loads half of the B tile
   bool ok = true;
   if (routed) {
     ok &= make_tmap(&a1r, x_perm, H, (uint64_t)budget, 0, H, 0, kBM);
     ok &= make_tmap(&b1r, W13, H, 2 * I, (uint64_t)s->N, H, 2 * I * H, kUmmaN / 2);
     ok &= make_tmap(&a2r, h, I, (uint64_t)budget, 0, I, 0, kBM);
-    ok &= make_tmap(&b2r, W2, I, H, (uint64_t)s->N, I, H * I, kUmmaN);
+    ok &= make_tmap(&b2r, W2, I, H, (uint64_t)s->N, I, H * I, b2_box);
   }
   if (shared) {
     const uint64_t S = s->S;
     ok &= make_tmap(&a1s, x_shared, H, (uint64_t)s->T, 0, H, 0, kBM);
     ok &= make_tmap(&b1s, Wsh13, H, 2 * I, S, H, 2 * I * H, kUmmaN / 2);
     ok &= make_tmap(&a2s, h_sh, S * I, (uint64_t)s->T, 0, S * I, 0, kBM);
-    ok &= make_tmap(&b2s, Wsh2, I, H, S, I, H * I, kUmmaN);
+    ok &= make_tmap(&b2s, Wsh2, I, H, S, I, H * I, b2_box);
   }
   if (!ok) return MOE_ERR_CUDA;
   if (!routed) { a1r = a1s; b1r = b1s; a2r = a2s; b2r = b2s; }
@@ -446,8 +723,9 @@ moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t*
   p.out_shared = reinterpret_cast<__nv_bfloat16*>(h_sh);
   p.ld_out_routed = s->I;
   p.ld_out_shared = (long long)s->S * s->I;
-  moe_status st = tile_n == 128 ? launch_gemm<true, 128>(p, a1r, b1r, a1s, b1s, stream)
-                                : launch_gemm<true, 256>(p, a1r, b1r, a1s, b1s, stream);
+  moe_status st = pairs           ? launch_gemm_pair<true>(p, a1r, b1r, a1s, b1s, stream)
+                  : tile_n == 128 ? launch_gemm<true, 128>(p, a1r, b1r, a1s, b1s, stream)
+                                  : launch_gemm<true, 256>(p, a1r, b1r, a1s, b1s, stream);
   if (st != MOE_OK) return st;
   if (between != nullptr) cudaEventRecord(between, stream);
   // GEMM-2
@@ -458,6 +736,7 @@ moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t*
   p.out_shared = reinterpret_cast<__nv_bfloat16*>(y_shared);
   p.ld_out_routed = s->H;
   p.ld_out_shared = s->H;
+  if (pairs) return launch_gemm_pair<false>(p, a2r, b2r, a2s, b2s, stream);
   return tile_n == 128 ? launch_gemm<false, 128>(p, a2r, b2r, a2s, b2s, stream)
                        : launch_gemm<false, 256>(p, a2r, b2r, a2s, b2s, stream);
 }

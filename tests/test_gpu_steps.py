@@ -282,3 +282,20 @@ def test_combine_against_oracle_formula():
     # one bf16 rounding of an fp32 sum of exactly representable products
     assert np.abs(got - want).max() <= 2 ** -8 * np.abs(want).max()
     assert max_rel(got, want) <= 4e-3
+
+
+@pytest.mark.parametrize("pair", ["0", "1"])
+def test_expert_gemm_variants_forced(pair):
+    """The library picks one-CTA or CTA-pair tiles by shape; both must be right on every shape.  The choice is read
+    from the environment once per process, so each forced setting runs the expert-GEMM tests in a process of its own."""
+    import os
+    import subprocess
+    import sys
+    if os.environ.get("ALLOCMOE_PAIR") is not None:
+        pytest.skip("already inside a forced run")
+    env = dict(os.environ, ALLOCMOE_PAIR=pair)
+    here = os.path.dirname(os.path.abspath(__file__))
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(here, "test_gpu_steps.py"), "-m", "gpu", "-q", "-x",
+                        "-k", "grouped_ffn or shared_ffn"], env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
