@@ -24,6 +24,14 @@ if ROOT not in sys.path:
 
 METRIC = "budgeted MoE-layer tokens/s"
 UNIT = "tokens/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel (expert GEMM-1), from the ncu
+# captures summarised under profiles/ (workload, budget) -> bytes; absent = not captured for the current kernel.
+NCU_TRAFFIC_BYTES = {
+    ("c2", 192): 717.5e6 + 4.7e6,        # profiles/ffn_gemm_c2_decode.md
+    ("c3", 12288): 833.3e6 + 37.4e6,     # profiles/ffn_gemm_c3_prefill.md
+}
+
+
 def kernels_per_layer(T):
     """Launches of one moe_layer_forward call: gate, routing (one fused launch up to 1024 tokens, else
     select + permute count/scan/place), row gather, 2 expert GEMMs, combine."""
@@ -355,8 +363,10 @@ def run_ours(args):
             roof = {"bound": "tensor", "achieved": g_flops / t_g1 / 1e12, "peak": peaks["bf16_tflops_sustained"],
                     "unit": "TFLOP/s"}
         roof["frac"] = roof["achieved"] / roof["peak"]
-        roof["traffic"] = None
-        roof["kernel"] = "ffn_gemm_kernel<true> (expert GEMM-1 + SwiGLU, routed and shared groups)"
+        roof["traffic"] = NCU_TRAFFIC_BYTES.get((cfg.name, int(budgets[0]))) if n_layers == 1 else None
+        pair = 128 * cfg.N < b_mean <= 256 * cfg.N      # the library's own rule for CTA-pair tiles
+        roof["kernel"] = ("ffn_gemm_pair_kernel<true>" if pair else "ffn_gemm_kernel<true, 256>") + \
+            " (expert GEMM-1 + SwiGLU, routed and shared groups)"
         roof["peak_source"] = peaks["source"] + (" (sustained bf16)" if roof["bound"] == "tensor" else " (copy)")
         roof["avg_launch_ms"] = stage_ms["ffn_gemm1"]
         roof["algorithmic_bytes"] = g_bytes
