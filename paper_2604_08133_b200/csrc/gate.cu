@@ -2,14 +2,14 @@
 // and the K_orig largest scores per token sorted descending (ties: lower expert id first).
 //
 // The contraction is small (2*T*H*N flops; 1 GFLOP at T=4096, H=2048, N=64) and x is read once,
-// so the kernel is bound by streaming x from HBM and, at decode sizes, by latency.  A CTA owns 32
-// tokens, all N experts and every KS-th chunk of 128 along H; the KS CTAs that share a token tile
-// form a thread-block cluster (KS = 8 for H >= 1024), so that T = 64 tokens still put 16 CTAs to
-// work and no CTA walks more than a few chunks.  Chunks of x and W_gate are staged in shared
-// memory with 16-byte cp.async (3 stages) and multiplied with mma.sync m16n8k16 bf16 -> fp32; the
-// four warps split every chunk's k-steps.  Partial logits are then added in a fixed order -- warps
-// 0..3 inside a CTA, CTAs 0..KS-1 of the cluster through distributed shared memory -- and each
-// CTA finishes softmax and Top-K for its 32/KS tokens.  W_gate is stored [H,N] (N contiguous, the
+// so the kernel is bound by streaming x from HBM and, at decode sizes, by latency.  A CTA owns
+// 16*NW tokens (one warp per 16 tokens; NW = 2 for small batches, 4 from 2048 tokens on, which
+// halves the re-reads of W_gate from L2), all N experts and every KS-th chunk of 128 along H; the
+// KS CTAs that share a token tile form a thread-block cluster (KS <= 8), so that T = 64 tokens
+// still put 16 CTAs to work and no CTA walks more than a few chunks.  Chunks of x and W_gate are
+// staged in shared memory with 16-byte cp.async (3 stages) and multiplied with mma.sync m16n8k16
+// bf16 -> fp32.  The KS partial logits of a token are then added in rank order through
+// distributed shared memory, and each CTA finishes softmax and Top-K for its 16*NW/KS tokens.  W_gate is stored [H,N] (N contiguous, the
 // paper's R^{H x N}), which is the "column" operand of mma.sync when read with ldmatrix.trans.
 #include <cooperative_groups.h>
 
@@ -19,10 +19,8 @@ namespace cg = cooperative_groups;
 
 namespace allocmoe {
 
-constexpr int kGateTM = 32;        // tokens per CTA
 constexpr int kGateKC = 128;       // H chunk
 constexpr int kGateStages = 3;
-constexpr int kGateThreads = 128;
 constexpr int kGateXStride = kGateKC + 8;   // bf16 elements per staged x row (272 B: conflict-free ldmatrix)
 
 DEV void ldmatrix_x4(uint32_t (&r)[4], const void* p) {
@@ -39,9 +37,9 @@ DEV void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// NT16 = number of 16-wide expert tiles (N padded to 16*NT16).
-template <int NT16>
-__global__ void __launch_bounds__(kGateThreads)
+// NT16 = number of 16-wide expert tiles (N padded to 16*NT16); NW = warps = 16-token slabs per CTA.
+template <int NT16, int NW>
+__global__ void __launch_bounds__(32 * NW)
 moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ W_gate,
                 const float* __restrict__ gate_bias, int T, int H, int N, int K_orig, int w_stride,
                 float* __restrict__ scores, int32_t* __restrict__ topk_idx, float* __restrict__ topk_score) {
@@ -49,6 +47,7 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
   const int KS = (int)cluster.num_blocks();        // CTAs per token tile (cluster spans blockIdx.y)
   const int ks_rank = (int)cluster.block_rank();
   constexpr int NP = NT16 * 16;
+  constexpr int kGateTM = 16 * NW, kGateThreads = 32 * NW;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int x_stage_bytes = kGateTM * kGateXStride * 2;
   const int w_stage_bytes = kGateKC * w_stride * 2;
@@ -82,13 +81,11 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
     cp_async_commit();
   };
 
-  float acc[2][NT16 * 2][4];
+  float acc[NT16 * 2][4];   // this warp's 16 tokens x NP experts
 #pragma unroll
-  for (int m = 0; m < 2; ++m)
+  for (int n = 0; n < NT16 * 2; ++n)
 #pragma unroll
-    for (int n = 0; n < NT16 * 2; ++n)
-#pragma unroll
-      for (int q = 0; q < 4; ++q) acc[m][n][q] = 0.f;
+    for (int q = 0; q < 4; ++q) acc[n][q] = 0.f;
 
   issue(0);
   issue(1);
@@ -100,21 +97,16 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
     const __nv_bfloat16* xs = reinterpret_cast<const __nv_bfloat16*>(st);
     const __nv_bfloat16* ws = reinterpret_cast<const __nv_bfloat16*>(st + x_stage_bytes);
 #pragma unroll
-    for (int ks = 0; ks < 2; ++ks) {
-      const int kk = (warp * 2 + ks) * 16;   // this warp's k-step inside the chunk
-      uint32_t a[2][4];
-#pragma unroll
-      for (int m = 0; m < 2; ++m)
-        ldmatrix_x4(a[m], xs + (m * 16 + (lane & 15)) * kGateXStride + kk + (lane >> 4) * 8);
+    for (int ks = 0; ks < kGateKC / 16; ++ks) {
+      const int kk = ks * 16;
+      uint32_t a[4];
+      ldmatrix_x4(a, xs + (warp * 16 + (lane & 15)) * kGateXStride + kk + (lane >> 4) * 8);
 #pragma unroll
       for (int n16 = 0; n16 < NT16; ++n16) {
         uint32_t b[4];
         ldmatrix_x4_trans(b, ws + (kk + (lane & 7) + ((lane >> 3) & 1) * 8) * w_stride + n16 * 16 + (lane >> 4) * 8);
-#pragma unroll
-        for (int m = 0; m < 2; ++m) {
-          mma_bf16_16816(acc[m][n16 * 2], a[m], b[0], b[1]);
-          mma_bf16_16816(acc[m][n16 * 2 + 1], a[m], b[2], b[3]);
-        }
+        mma_bf16_16816(acc[n16 * 2], a, b[0], b[1]);
+        mma_bf16_16816(acc[n16 * 2 + 1], a, b[2], b[3]);
       }
     }
     __syncthreads();
@@ -122,32 +114,21 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
   cp_async_wait<0>();
   __syncthreads();
 
-  // Cross-warp sum in a fixed order.  red[w][row][col], fp32, aliasing the staging buffers.
+  // This CTA's partial logits: red[row][col], fp32, aliasing the staging buffers.
   float* red = reinterpret_cast<float*>(smem_raw);
   constexpr int RS = NP + 1;
   {
     const int g = lane >> 2, tq = lane & 3;
 #pragma unroll
-    for (int m = 0; m < 2; ++m)
-#pragma unroll
-      for (int n = 0; n < NT16 * 2; ++n) {
-        float* base = red + ((warp * kGateTM + m * 16 + g) * RS + n * 8 + tq * 2);
-        base[0] = acc[m][n][0];
-        base[1] = acc[m][n][1];
-        base[8 * RS] = acc[m][n][2];
-        base[8 * RS + 1] = acc[m][n][3];
-      }
+    for (int n = 0; n < NT16 * 2; ++n) {
+      float* base = red + ((warp * 16 + g) * RS + n * 8 + tq * 2);
+      base[0] = acc[n][0];
+      base[1] = acc[n][1];
+      base[8 * RS] = acc[n][2];
+      base[8 * RS + 1] = acc[n][3];
+    }
   }
-  __syncthreads();
-  for (int i = tid; i < kGateTM * NP; i += kGateThreads) {
-    const int r = i / NP, c = i % NP;
-    float v = red[(0 * kGateTM + r) * RS + c];
-    v += red[(1 * kGateTM + r) * RS + c];
-    v += red[(2 * kGateTM + r) * RS + c];
-    v += red[(3 * kGateTM + r) * RS + c];
-    red[r * RS + c] = v;   // row r of warp block 0: each (r,c) is read and written by this thread only
-  }
-  cluster.sync();   // every CTA's partial logits are in its red[0 .. 32*RS)
+  cluster.sync();   // every CTA's partial logits are in its red[0 .. 16*NW*RS)
 
   // Softmax and sorted Top-K_orig.  This CTA finishes tokens ks_rank*32/KS .. of the tile, one warp
   // per token at a time; lane l owns experts l, l+32, ...  The KS partial sums are added in rank
@@ -157,7 +138,7 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
   const float* rred[8];
 #pragma unroll
   for (int k = 0; k < 8; ++k) rred[k] = cluster.map_shared_rank(red, k < KS ? k : 0);
-  for (int rr = warp; rr < rows_per; rr += kGateThreads / 32) {
+  for (int rr = warp; rr < rows_per; rr += NW) {
     const int r = ks_rank * rows_per + rr;
     const int t = t0 + r;
     if (t >= T) continue;   // uniform across the warp
@@ -228,45 +209,53 @@ static int gate_w_stride(int NP) {
   return s16 * 8;
 }
 
-template <int NT16>
+template <int NT16, int NW>
 static moe_status gate_launch_t(const moe_shape* s, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,
                                 float* scores, int32_t* topk_idx, float* topk_score, cudaStream_t stream) {
-  constexpr int NP = NT16 * 16;
+  constexpr int NP = NT16 * 16, TM = 16 * NW;
   const int w_stride = gate_w_stride(NP);
-  size_t pipe = (size_t)kGateStages * (kGateTM * kGateXStride * 2 + kGateKC * w_stride * 2);
-  size_t red = (size_t)4 * kGateTM * (NP + 1) * 4;
+  size_t pipe = (size_t)kGateStages * (TM * kGateXStride * 2 + kGateKC * w_stride * 2);
+  size_t red = (size_t)TM * (NP + 1) * 4;
   size_t smem = pipe > red ? pipe : red;
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(moe_gate_kernel<NT16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(moe_gate_kernel<NT16, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
       return MOE_ERR_CUDA;
     attr_done = true;
   }
   // CTAs per token tile: a power of two <= 8 that leaves every CTA at least one chunk, grown until
   // the grid has about two CTAs per SM (more only adds cluster barriers)
   const int nchunks = (s->H + kGateKC - 1) / kGateKC;
-  const int tiles = (s->T + kGateTM - 1) / kGateTM;
+  const int tiles = (s->T + TM - 1) / TM;
   int ks = 1;
   while (ks * 2 <= 8 && ks * 2 <= nchunks && tiles * ks < 296) ks *= 2;
   const cudaError_t err = launch_dependent(
-      moe_gate_kernel<NT16>, dim3((unsigned)tiles, (unsigned)ks, 1), dim3(kGateThreads), smem, stream, (unsigned)ks,
+      moe_gate_kernel<NT16, NW>, dim3((unsigned)tiles, (unsigned)ks, 1), dim3(32 * NW), smem, stream, (unsigned)ks,
       reinterpret_cast<const __nv_bfloat16*>(x), reinterpret_cast<const __nv_bfloat16*>(W_gate), gate_bias, (int)s->T,
       (int)s->H, (int)s->N, (int)s->K_orig, w_stride, scores, topk_idx, topk_score);
   return err == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+template <int NT16>
+static moe_status gate_launch_nw(const moe_shape* s, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,
+                                 float* scores, int32_t* topk_idx, float* topk_score, cudaStream_t stream) {
+  if (s->T >= 2048) return gate_launch_t<NT16, 4>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+  return gate_launch_t<NT16, 2>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
 }
 
 moe_status launch_moe_gate(const moe_shape* s, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,
                            float* scores, int32_t* topk_idx, float* topk_score, cudaStream_t stream) {
   const int nt16 = (s->N + 15) / 16;
   switch (nt16) {
-    case 1: return gate_launch_t<1>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-    case 2: return gate_launch_t<2>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-    case 3: return gate_launch_t<3>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-    case 4: return gate_launch_t<4>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-    case 5: return gate_launch_t<5>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-    case 6: return gate_launch_t<6>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-    case 7: return gate_launch_t<7>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-    case 8: return gate_launch_t<8>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 1: return gate_launch_nw<1>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 2: return gate_launch_nw<2>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 3: return gate_launch_nw<3>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 4: return gate_launch_nw<4>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 5: return gate_launch_nw<5>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 6: return gate_launch_nw<6>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 7: return gate_launch_nw<7>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 8: return gate_launch_nw<8>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
     default: return MOE_ERR_ARG;
   }
 }
