@@ -236,6 +236,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2604_08133_b200 import binding as B
+    from paper_2604_08133_b200 import dist as pdist
     from paper_2604_08133_b200 import synth
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -300,12 +301,7 @@ def run_ours(args):
             fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return pdist.max_over_ranks(e0.elapsed_time(e1), device="cuda")
 
     for _ in range(warmup):
         step()

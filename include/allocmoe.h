@@ -186,6 +186,18 @@ moe_status moe_layer_intermediates(const moe_shape* shape, int64_t budget, void*
                                    int32_t** n_sel, int32_t** expert_offsets,
                                    int32_t** perm_token, int32_t** pair_pos, uint16_t** y_perm);
 
+/* Alloc-L, the layer-level allocation (Sec. 3.2, Eq. 3-6): K_i in 1..K_orig per layer minimising
+ * sum_i S[i, K_i] subject to sum_i K_i <= B, solved exactly by the grouped-knapsack dynamic
+ * programme of Eq. 6 with backtracking.  Host code, run once off line; no GPU involved.
+ *   S        host fp64 [L, K_orig] row-major; S[i, k-1] is the sensitivity cost of giving layer i
+ *            k experts per token (the paper's S[i, k]); must be finite
+ *   B        global budget per token; B < L returns MOE_ERR_BUDGET (Eq. 5 infeasible)
+ *   K_out    host int32 [L]: the optimal allocation (ties: the smaller k, then the smaller total)
+ *   cost_out host fp64 [1] or NULL: its total cost
+ * K_orig <= 255.  MOE_ERR_WORKSPACE if the host cannot allocate the L * (min(B, L*K_orig) + 1)
+ * bytes of backtracking state. */
+moe_status alloc_l_solve(const double* S, int32_t L, int32_t K_orig, int64_t B, int32_t* K_out, double* cost_out);
+
 /* Instrumentation (no counterpart in the paper): with profiling on, moe_layer_forward records
  * CUDA events at its stage boundaries; moe_profile_read waits for the last forward call and
  * returns the device time in milliseconds of its 6 stages: gate, alloc_t_select, moe_permute,

@@ -16,7 +16,7 @@ MOE_OK, MOE_ERR_ARG, MOE_ERR_BUDGET, MOE_ERR_WORKSPACE, MOE_ERR_CUDA, MOE_ERR_NO
 
 EXPORTS = ("moe_status_string", "moe_workspace_bytes", "moe_gate", "alloc_t_select", "moe_permute",
            "moe_grouped_ffn", "moe_shared_ffn", "moe_combine", "moe_layer_forward", "moe_layer_intermediates",
-           "moe_rmsnorm", "moe_profile_enable", "moe_profile_read", "moe_permute_static", "moe_route")
+           "moe_rmsnorm", "moe_profile_enable", "moe_profile_read", "moe_permute_static", "moe_route", "alloc_l_solve")
 PROFILE_STAGES = ("gate", "select", "permute", "ffn_gemm1", "ffn_gemm2", "combine")
 
 
@@ -64,6 +64,9 @@ def lib() -> ctypes.CDLL:
             "moe_profile_enable": [ctypes.c_int32],
             "moe_profile_read": [ctypes.POINTER(ctypes.c_float)],
         }
+        L.alloc_l_solve.restype = ctypes.c_int
+        L.alloc_l_solve.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.c_int32, ctypes.c_int32, i64,
+                                    ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_double)]
         for name, argtypes in sigs.items():
             fn = getattr(L, name)
             fn.restype = ctypes.c_int
@@ -129,6 +132,18 @@ def moe_permute(shape, x, topk_idx, topk_score, n_sel, budget, expert_offsets, p
                                             int(budget), _p(expert_offsets), _p(perm_token), _p(perm_weight),
                                             _p(pair_pos), _p(x_perm), _p(dev_status), _p(ws), ws.numel(),
                                             _stream(stream)))
+
+
+def alloc_l_solve(S, B: int):
+    """Alloc-L (Eq. 3-6): the optimal per-layer K for a sensitivity matrix S [L, K_orig] (any array-like of floats)
+    under the global budget B.  Returns (list of K_i, total cost).  Host only."""
+    rows = [[float(v) for v in r] for r in S]
+    Lr, K = len(rows), len(rows[0])
+    flat = (ctypes.c_double * (Lr * K))(*[v for r in rows for v in r])
+    out = (ctypes.c_int32 * Lr)()
+    cost = ctypes.c_double(0.0)
+    _check("alloc_l_solve", lib().alloc_l_solve(flat, Lr, K, int(B), out, ctypes.byref(cost)))
+    return list(out), float(cost.value)
 
 
 def moe_route(shape, topk_idx, topk_score, budget, n_sel, expert_offsets, perm_token, perm_weight, pair_pos, dev_status,

@@ -13,7 +13,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "liballocmoe.so")
-SOURCES = ["api.cu", "gate.cu", "select.cu", "permute.cu", "route.cu", "ffn.cu", "combine.cu"]
+SOURCES = ["api.cu", "gate.cu", "select.cu", "permute.cu", "route.cu", "ffn.cu", "combine.cu", "alloc_l.cpp"]
 
 
 def _nvcc() -> str:

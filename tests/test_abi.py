@@ -21,7 +21,7 @@ def lib():
 def _declared():
     with open(os.path.join(ROOT, "include", "allocmoe.h")) as f:
         src = re.sub(r"/\*.*?\*/", "", f.read(), flags=re.S)
-    return sorted(set(re.findall(r"\b(moe_[a-z_0-9]+|alloc_t_select)\s*\(", src)))
+    return sorted(set(re.findall(r"\b(moe_[a-z_0-9]+|alloc_t_select|alloc_l_solve)\s*\(", src)))
 
 
 def test_every_declared_symbol_is_exported(lib):

@@ -203,3 +203,22 @@ def test_c4_stack_teacher_forced():
         assert 0.5 < float(out.float().std()) < 50.0          # the pre-norm stream grows slowly
         x = out
         del d
+
+
+def test_global_selection_path_equals_the_fused_call_on_one_rank():
+    """With one rank the batch-wide selection is the local one: the step-by-step path of dist.py (gate, selection,
+    permute, experts, combine as separate C-ABI calls) must give the fused call's output bit for bit."""
+    from paper_2604_08133_b200 import dist as D
+    cfg = synth.CONFIGS["c2"]
+    d = dev_layer(cfg)
+    out_fused, inter, status = forward_gpu(cfg, d)
+    assert status == 0
+    shape = B.shape_of(cfg)
+    out = torch.empty_like(d["x"])
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    b_local = D.moe_layer_forward_global(shape, d["x"], d["W_gate"], d["gate_bias"], d["W13"], d["W2"], d["Wsh13"],
+                                         d["Wsh2"], cfg.budget, out, st)
+    torch.cuda.synchronize()
+    assert st.item() == 0 and b_local == cfg.budget
+    assert torch.equal(out, out_fused)
+
