@@ -51,7 +51,7 @@ typedef enum {
 
 /* T tokens, H hidden size, N routed experts, I expert intermediate size, S shared experts,
  * K_orig nominal Top-K (candidates per token), K_base guaranteed experts per token (Eq. 10).
- * Supported: H % 64 == 0, I % 64 == 0, 8 <= N <= 128 with N % 8 == 0, 1 <= K_orig <= min(N, 16),
+ * Supported: H % 64 == 0, I % 64 == 0, 8 <= N <= 128 with N % 4 == 0, 1 <= K_orig <= min(N, 16),
  * 0 <= K_base <= K_orig, S >= 0, T >= 1, T*K_orig < 2^31.  flags must be 0. */
 typedef struct {
   int32_t T, H, N, I, S, K_orig, K_base;

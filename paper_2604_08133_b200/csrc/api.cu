@@ -29,7 +29,7 @@ bool shape_ok(const moe_shape* s) {
   if (s == nullptr) return false;
   if (s->flags != 0) return false;
   if (s->T < 1 || s->H < 64 || s->I < 64 || s->N < 8 || s->S < 0) return false;
-  if (s->H % 64 != 0 || s->I % 64 != 0 || s->N % 8 != 0 || s->N > 128) return false;
+  if (s->H % 64 != 0 || s->I % 64 != 0 || s->N % 4 != 0 || s->N > 128) return false;
   if (s->K_orig < 1 || s->K_orig > 16 || s->K_orig > s->N) return false;
   if (s->K_base < 0 || s->K_base > s->K_orig) return false;
   if ((long long)s->T * s->K_orig >= (1ll << 31)) return false;

@@ -71,11 +71,20 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
         const bool ok = (t < T) && (k < H);
         cp_async_16(xs + r * kGateXStride + c * 8, x + (ok ? ((long long)t * H + k) : 0), ok);
       }
-      for (int i = tid; i < kGateKC * (NP / 8); i += kGateThreads) {
-        const int r = i / (NP / 8), c = i % (NP / 8);
-        const int k = k0 + r;
-        const bool ok = (k < H) && (c < n_vec);
-        cp_async_16(ws + r * w_stride + c * 8, W_gate + (ok ? ((long long)k * N + c * 8) : 0), ok);
+      if ((N & 7) == 0) {
+        for (int i = tid; i < kGateKC * (NP / 8); i += kGateThreads) {
+          const int r = i / (NP / 8), c = i % (NP / 8);
+          const int k = k0 + r;
+          const bool ok = (k < H) && (c < n_vec);
+          cp_async_16(ws + r * w_stride + c * 8, W_gate + (ok ? ((long long)k * N + c * 8) : 0), ok);
+        }
+      } else {   // N a multiple of 4 only: rows of W_gate start on 8-byte boundaries
+        for (int i = tid; i < kGateKC * (NP / 4); i += kGateThreads) {
+          const int r = i / (NP / 4), c = i % (NP / 4);
+          const int k = k0 + r;
+          const bool ok = (k < H) && (c < N / 4);
+          cp_async_8(ws + r * w_stride + c * 4, W_gate + (ok ? ((long long)k * N + c * 4) : 0), ok);
+        }
       }
     }
     cp_async_commit();

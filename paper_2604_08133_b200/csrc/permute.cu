@@ -140,7 +140,7 @@ extern "C" moe_status moe_permute_static(const moe_shape* shape, const uint16_t*
                                          int32_t* expert_offsets, int32_t* perm_token, float* perm_weight,
                                          int32_t* pair_pos, uint16_t* x_perm, int32_t* dev_status, void* stream) {
   const moe_shape* s = shape;
-  if (s == nullptr || s->flags != 0 || s->T < 1 || s->H < 64 || s->H % 64 != 0 || s->N < 8 || s->N % 8 != 0 ||
+  if (s == nullptr || s->flags != 0 || s->T < 1 || s->H < 64 || s->H % 64 != 0 || s->N < 8 || s->N % 4 != 0 ||
       s->N > kMaxExperts || s->K_orig < 1 || s->K_orig > 16 || s->K_orig > s->N || s->K_base < 0 ||
       s->K_base > s->K_orig || (long long)s->T * s->K_orig >= (1ll << 31))
     return MOE_ERR_ARG;

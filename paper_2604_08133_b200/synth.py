@@ -162,6 +162,11 @@ CONFIGS: Dict[str, MoEConfig] = {
     # large-expert layer, prefill.
     "c5": MoEConfig("c5", T=8192, H=4096, N=8, I=14336, S=0, K_orig=2, K_base=1, budget=12288,
                     gate_scale=C5_GATE_SCALE),
+    # the other two model rows of the paper's Table 1, prefill: Qwen1.5-MoE-shaped (60 routed experts, Top-4, budgets
+    # 2-3.5 per token) and OLMoE-shaped (64 routed experts, Top-8, budgets 4-7).  The paper gives the expert counts
+    # and Top-K only; hidden and intermediate sizes and the shared expert are synthetic choices.
+    "qwen": MoEConfig("qwen", T=4096, H=2048, N=60, I=1408, S=1, K_orig=4, K_base=1, budget=int(2.5 * 4096)),
+    "olmoe": MoEConfig("olmoe", T=4096, H=2048, N=64, I=1024, S=0, K_orig=8, K_base=1, budget=5 * 4096),
 }
 
 C3_BUDGET_MULTS = (6.0, 4.5, 3.0, 2.0)

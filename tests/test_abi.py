@@ -46,7 +46,7 @@ def test_workspace_bytes_is_host_only_and_monotone(lib):
     # x_perm + h + y_perm dominate: budget * (2H + I) * 2 bytes
     assert b >= 6 * 4096 * (2 * 2048 + 1408) * 2
     assert B.moe_workspace_bytes(s, 6 * 4096 + 1) == 0            # beyond K_orig*T
-    for bad in (B.make_shape(64, 100, 64, 1408, 0, 6, 1), B.make_shape(64, 2048, 60, 1408, 0, 6, 1),
+    for bad in (B.make_shape(64, 100, 64, 1408, 0, 6, 1), B.make_shape(64, 2048, 62, 1408, 0, 6, 1),
                 B.make_shape(64, 2048, 64, 1408, 0, 6, 7), B.make_shape(0, 2048, 64, 1408, 0, 6, 1),
                 B.make_shape(64, 2048, 8, 1408, 0, 9, 1)):
         assert B.moe_workspace_bytes(bad, 64) == 0

@@ -222,3 +222,11 @@ def test_global_selection_path_equals_the_fused_call_on_one_rank():
     assert st.item() == 0 and b_local == cfg.budget
     assert torch.equal(out, out_fused)
 
+
+@pytest.mark.parametrize("name,T,mult", [("qwen", 320, 2.5), ("qwen", 320, 3.5), ("olmoe", 256, 5.0), ("olmoe", 256, 7.0)])
+def test_other_model_shapes(name, T, mult):
+    """Qwen1.5-MoE-shaped (60 experts: not a multiple of 8, Top-4) and OLMoE-shaped (Top-8: a residual pool seven
+    columns wide) layers at a size the oracle finishes in seconds."""
+    cfg = synth.CONFIGS[name].with_(T=T, budget=int(mult * T))
+    _full_check(cfg)
+
