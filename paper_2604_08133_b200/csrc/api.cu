@@ -16,7 +16,8 @@ moe_status launch_moe_route(const moe_shape*, const float*, const int32_t*, int6
                             int32_t*, int32_t*, cudaStream_t);
 moe_status launch_ffn(const moe_shape*, const uint16_t*, const int32_t*, int64_t, const uint16_t*, const uint16_t*,
                       uint16_t*, uint16_t*, const uint16_t*, const uint16_t*, const uint16_t*, uint16_t*, uint16_t*,
-                      int32_t*, cudaStream_t, cudaEvent_t);
+                      int32_t*, int32_t*, cudaStream_t, cudaEvent_t);
+size_t ffn_done_ints(const moe_shape*, int64_t);
 moe_status launch_moe_combine(const moe_shape*, const uint16_t*, const int32_t*, const float*, const int32_t*,
                               const uint16_t*, const uint16_t*, long long, uint16_t*, cudaStream_t);
 moe_status launch_rmsnorm(const moe_shape*, const uint16_t*, uint16_t*, cudaStream_t);
@@ -43,7 +44,7 @@ bool budget_ok(const moe_shape* s, int64_t budget) {
 // Fixed carve-up of the workspace; every region starts on a 256-byte boundary.
 struct WsLayout {
   size_t topk_idx, topk_score, n_sel, expert_offsets, perm_token, perm_weight, pair_pos, seg_counts;
-  size_t x_perm, h, y_perm, h_sh, y_shared, total;
+  size_t x_perm, h, y_perm, h_sh, y_shared, gemm_done, total;
 };
 
 WsLayout ws_layout(const moe_shape* s, int64_t budget_max) {
@@ -68,6 +69,7 @@ WsLayout ws_layout(const moe_shape* s, int64_t budget_max) {
   L.y_perm = take(B * H * 2);
   L.h_sh = take(T * S * I * 2);
   L.y_shared = take(T * H * 2);
+  L.gemm_done = take(ffn_done_ints(s, budget_max) * 4);
   L.total = off;
   return L;
 }
@@ -160,7 +162,7 @@ moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_perm, const
   const WsLayout L = ws_layout(shape, budget);
   if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
   return launch_ffn(shape, x_perm, expert_offsets, budget, W13, W2, at<uint16_t>(ws, L.h), y_perm, nullptr, nullptr,
-                    nullptr, nullptr, nullptr, dev_status, (cudaStream_t)stream, nullptr);
+                    nullptr, nullptr, nullptr, dev_status, at<int32_t>(ws, L.gemm_done), (cudaStream_t)stream, nullptr);
 }
 
 moe_status moe_shared_ffn(const moe_shape* shape, const uint16_t* x, const uint16_t* Wsh13, const uint16_t* Wsh2,
@@ -170,7 +172,8 @@ moe_status moe_shared_ffn(const moe_shape* shape, const uint16_t* x, const uint1
   const WsLayout L = ws_layout(shape, 0);
   if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
   return launch_ffn(shape, nullptr, nullptr, 0, nullptr, nullptr, nullptr, nullptr, x, Wsh13, Wsh2,
-                    at<uint16_t>(ws, L.h_sh), y_shared, dev_status, (cudaStream_t)stream, nullptr);
+                    at<uint16_t>(ws, L.h_sh), y_shared, dev_status, at<int32_t>(ws, L.gemm_done), (cudaStream_t)stream,
+                    nullptr);
 }
 
 moe_status moe_combine(const moe_shape* shape, const uint16_t* y_perm, const int32_t* pair_pos,
@@ -228,8 +231,8 @@ moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const ui
   if (r != MOE_OK) return r;
   prof_mark(3, st);
   r = launch_ffn(shape, x_perm, expert_offsets, budget, W13, W2, at<uint16_t>(ws, L.h), y_perm,
-                 shape->S > 0 ? x : nullptr, Wsh13, Wsh2, at<uint16_t>(ws, L.h_sh), y_shared, dev_status, st,
-                 g_prof_on ? g_prof_ev[4] : nullptr);
+                 shape->S > 0 ? x : nullptr, Wsh13, Wsh2, at<uint16_t>(ws, L.h_sh), y_shared, dev_status,
+                 at<int32_t>(ws, L.gemm_done), st, g_prof_on ? g_prof_ev[4] : nullptr);
   if (r != MOE_OK) return r;
   prof_mark(5, st);
   r = launch_moe_combine(shape, y_perm, pair_pos, topk_score, n_sel, y_shared, residual, budget, out,

@@ -30,6 +30,47 @@ DEV void pdl_prologue_done() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+constexpr long long kWaitLimitClk = 1000ll * 1000ll * 1000ll;   // bounded waits: about 0.5 s at 1.9 GHz
+DEV void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+DEV void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// ------------------------------------------------------------------ flags between kernels / CTAs
+// A tile of h written with ordinary stores by GEMM-1's epilogue is read by GEMM-2's TMA loads
+// (the async proxy), possibly while GEMM-1 is still running on other SMs.  Writer: stores,
+// __threadfence, barrier among the storing warps, then one thread fence_proxy_async_global +
+// flag_add_release.  Reader: flag_load_acquire until the count is reached, fence_proxy_async_global,
+// then the TMA loads.
+DEV void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
+DEV void flag_add_release(int32_t* flag, int v) {
+  asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(flag), "r"(v) : "memory");
+}
+DEV int flag_load_acquire(const int32_t* flag) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+  return v;
+}
+// Bounded wait for *flag >= need (same limit and abort protocol as the mbarrier waits).
+DEV bool flag_wait_bounded(const int32_t* flag, int need, volatile int* abort_flag, int32_t* dev_status) {
+  if (flag_load_acquire(flag) >= need) return true;
+  long long t0 = 0;
+  uint32_t spins = 0;
+  while (true) {
+    __nanosleep(64);
+    if (flag_load_acquire(flag) >= need) return true;
+    if ((++spins & 63u) == 0u) {
+      if (*abort_flag) return false;
+      const long long now = clock64();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > kWaitLimitClk) {
+        *abort_flag = 1;
+        set_dev_status(dev_status, MOE_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
 // ------------------------------------------------------------------ mbarrier
 DEV void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
@@ -57,7 +98,6 @@ DEV bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // then returns false at its next poll, the roles leave their loops and the CTA tears down
 // normally (drains its own copies, frees TMEM, returns).  Time is the SM's own cycle counter,
 // looked at only every 64th poll, so a wait that succeeds quickly never pays for it.
-constexpr long long kWaitLimitClk = 1000ll * 1000ll * 1000ll;   // about 0.5 s at 1.9 GHz
 constexpr long long kDrainLimitClk = 40ll * 1000ll * 1000ll;    // teardown waits: about 20 ms
 
 DEV bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {

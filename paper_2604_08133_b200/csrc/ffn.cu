@@ -55,6 +55,11 @@ struct FfnGemmParams {
   __nv_bfloat16* out_shared;        // GEMM-1: h_sh [T, S*I]; GEMM-2: y_shared [T, H]
   long long ld_out_routed, ld_out_shared;
   int32_t* dev_status;
+  // GEMM-2 may start while GEMM-1 is still running: per block of token rows, GEMM-1 counts the tiles
+  // of h it has finished (done[block], once per epilogue warp) and GEMM-2 loads a block's rows once
+  // the count reaches dep_need_* (GEMM-1's tiles per block x epilogue warps).  nullptr = no tracking.
+  int32_t* done;
+  int dep_need_routed, dep_need_shared;
 };
 
 struct FfnSmemCtl {
@@ -70,10 +75,12 @@ struct FfnSmemCtl {
   int tile_start[kMaxGroups + 1];   // first tile of each group
   int row_start[kMaxGroups];        // first row of each group in its A / output matrix
   int row_count[kMaxGroups];
+  int mblock_start[kMaxGroups + 1]; // first row block of each group in the numbering of `done`
 };
 
 struct TileCoord {
   int group, m0, m_end, nb;
+  int dep_id;       // index of the tile's row block in `done`
   bool shared;
 };
 
@@ -98,6 +105,7 @@ struct TileWalker {
     const int mblocks = (c->row_count[g] + kTileM - 1) / kTileM;
     tc.nb = local / mblocks;
     const int mb = local % mblocks;
+    tc.dep_id = c->mblock_start[g] + mb;
     tc.m0 = c->row_start[g] + mb * kTileM;
     tc.m_end = c->row_start[g] + c->row_count[g];
     return tc;
@@ -134,7 +142,11 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
     tmem_alloc(&ctl->tmem_base, kTmemCols);
     tmem_relinquish();
   }
-  pdl_prologue_done();   // expert_offsets and the operands come from earlier kernels of the stream
+  // GEMM-1 waits for everything before it and only then lets GEMM-2 start, so a GEMM-2 CTA that finds
+  // an SM free while GEMM-1 is in its last round sees complete routing data; GEMM-2 itself does not
+  // wait for the whole of GEMM-1 but for the row blocks of h it needs (p.done).
+  if (kSwiGLU || p.done == nullptr) pdl_wait();
+  pdl_launch_dependents();   // expert_offsets and the operands come from earlier kernels of the stream
   for (int gi = tid; gi < n_groups; gi += kFfnThreads) {
     if (gi < p.n_experts) {
       const int lo = p.expert_offsets[gi], hi = p.expert_offsets[gi + 1];
@@ -148,11 +160,13 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   __syncthreads();
   if (tid == 0) {
     TileWalker<kSwiGLU, kN, kBM> w(ctl, p);
-    int acc = 0;
+    int acc = 0, mb_acc = 0;
     for (int gi = 0; gi < n_groups; ++gi) {
       ctl->tile_start[gi] = acc;
+      ctl->mblock_start[gi] = mb_acc;
       const int mblocks = (ctl->row_count[gi] + kBM - 1) / kBM;
       acc += mblocks * (gi < p.n_experts ? w.nb_routed : w.nb_shared);
+      mb_acc += mblocks;
     }
     ctl->tile_start[n_groups] = acc;
     ctl->total_tiles = acc;
@@ -183,6 +197,12 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
         if (tc.shared) {
           if (kSwiGLU) { e_n = tc.nb / w.nb_routed; n_row = (tc.nb % w.nb_routed) * kOutCols; }
           else { e_n = 0; }
+        }
+        if (!kSwiGLU && p.done != nullptr) {   // the block's rows of h are complete?
+          if (!(ok = flag_wait_bounded(p.done + tc.dep_id, tc.shared ? p.dep_need_shared : p.dep_need_routed,
+                                       abort_flag, p.dev_status)))
+            break;
+          fence_proxy_async_global();
         }
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % kStages;
@@ -304,6 +324,14 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
           }
         }
       }
+      if (kSwiGLU && p.done != nullptr) {   // publish this warp's quarter of the tile (FfnGemmParams::done)
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) {
+          fence_proxy_async_global();
+          flag_add_release(p.done + tc.dep_id, 1);
+        }
+      }
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&ctl->tmem_empty[a]);
@@ -369,7 +397,11 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
     tmem_alloc_pair(&ctl->tmem_base, kTmemCols);
     tmem_relinquish_pair();
   }
-  pdl_prologue_done();
+  // GEMM-1 waits for everything before it and only then lets GEMM-2 start, so a GEMM-2 CTA that finds
+  // an SM free while GEMM-1 is in its last round sees complete routing data; GEMM-2 itself does not
+  // wait for the whole of GEMM-1 but for the row blocks of h it needs (p.done).
+  if (kSwiGLU || p.done == nullptr) pdl_wait();
+  pdl_launch_dependents();
   for (int gi = tid; gi < n_groups; gi += kFfnThreads) {
     if (gi < p.n_experts) {
       const int lo = p.expert_offsets[gi], hi = p.expert_offsets[gi + 1];
@@ -383,11 +415,13 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
   __syncthreads();
   if (tid == 0) {
     TileWalker<kSwiGLU, kN, kPairM> w(ctl, p);
-    int acc = 0;
+    int acc = 0, mb_acc = 0;
     for (int gi = 0; gi < n_groups; ++gi) {
       ctl->tile_start[gi] = acc;
+      ctl->mblock_start[gi] = mb_acc;
       const int mblocks = (ctl->row_count[gi] + kPairM - 1) / kPairM;
       acc += mblocks * (gi < p.n_experts ? w.nb_routed : w.nb_shared);
+      mb_acc += mblocks;
     }
     ctl->tile_start[n_groups] = acc;
     ctl->total_tiles = acc;
@@ -422,6 +456,12 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
         // this CTA's half of the B tile: GEMM-1 W1 rows (leader) or W3 rows (peer); GEMM-2 rows +128*rank
         const int b_row = kSwiGLU ? (rank == 0 ? n_row : p.up_row_offset + n_row) : n_row + (int)rank * (kN / 2);
         const int a_row = tc.m0 + (int)rank * kBM;
+        if (!kSwiGLU && p.done != nullptr) {   // the block's rows of h are complete?
+          if (!(ok = flag_wait_bounded(p.done + tc.dep_id, tc.shared ? p.dep_need_shared : p.dep_need_routed,
+                                       abort_flag, p.dev_status)))
+            break;
+          fence_proxy_async_global();
+        }
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % kPairStages;
           const uint32_t ph = (it / kPairStages) & 1u;
@@ -541,6 +581,14 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
                 reinterpret_cast<uint16_t*>(out_row)[col + i] = (uint16_t)((i & 1) ? (w2 >> 16) : (w2 & 0xFFFFu));
               }
           }
+        }
+      }
+      if (kSwiGLU && p.done != nullptr) {   // publish this warp's quarter of the tile (FfnGemmParams::done)
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) {
+          fence_proxy_async_global();
+          flag_add_release(p.done + tc.dep_id, 1);
         }
       }
       tc_fence_before_sync();
@@ -676,12 +724,17 @@ static int pick_tile_n(const moe_shape*, int64_t, bool) {
   return forced ? forced : 256;
 }
 
+// Ints of row-block counters a call needs: one per 128-row block of every group at most.
+size_t ffn_done_ints(const moe_shape* s, int64_t budget) {
+  return (size_t)(budget / kBM + s->N + (s->S > 0 ? s->T / kBM + 1 : 0) + 4);
+}
+
 // Routed and/or shared experts in one pair of launches.
 //   routed part present iff budget > 0 && x_perm != nullptr; shared part iff S > 0 && x_shared != nullptr.
 moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t* expert_offsets, int64_t budget,
                       const uint16_t* W13, const uint16_t* W2, uint16_t* h, uint16_t* y_perm, const uint16_t* x_shared,
                       const uint16_t* Wsh13, const uint16_t* Wsh2, uint16_t* h_sh, uint16_t* y_shared,
-                      int32_t* dev_status, cudaStream_t stream, cudaEvent_t between) {
+                      int32_t* dev_status, int32_t* done, cudaStream_t stream, cudaEvent_t between) {
   const bool routed = (budget > 0 && x_perm != nullptr);
   const bool shared = (s->S > 0 && x_shared != nullptr);
   if (!routed && !shared) return MOE_OK;
@@ -715,6 +768,16 @@ moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t*
   p.shared_rows = shared ? s->T : 0;
   p.shared_sub = s->S;
   p.dev_status = dev_status;
+  // row-block completion counters for the GEMM-1 -> GEMM-2 hand-over
+  p.done = done;
+  if (done != nullptr) {
+    const int nb1 = (int)((s->I + kUmmaN / 2 - 1) / (kUmmaN / 2));      // GEMM-1 column blocks per (sub-)expert
+    const int per_tile = 4 * (pairs ? 2 : 1);                           // every epilogue warp counts once
+    p.dep_need_routed = nb1 * per_tile;
+    p.dep_need_shared = nb1 * s->S * per_tile;
+    if (cudaMemsetAsync(done, 0, ffn_done_ints(s, routed ? budget : 0) * sizeof(int32_t), stream) != cudaSuccess)
+      return MOE_ERR_CUDA;
+  }
   // GEMM-1
   p.n_per_sub = s->I;
   p.k_per_sub = s->H;
