@@ -46,6 +46,10 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--budget-mult", type=float, default=None, help="budget as a multiple of T")
+    ap.add_argument("--k-base", type=int, default=None, help="override K_base (the guaranteed experts per token)")
+    ap.add_argument("--stack-budgets", default="dirichlet", choices=["dirichlet", "alloc-l"],
+                    help="layer stack only: per-layer budgets from the seeded Dirichlet split, or from alloc_l_solve "
+                         "on a seeded synthetic sensitivity matrix (same total)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the stage profile / full-Top-K / e2e passes")
     return ap.parse_args()
@@ -64,7 +68,10 @@ def load_peaks():
 def workload_cfg(args):
     from paper_2604_08133_b200 import synth
     cfg = synth.CONFIGS[args.workload]
+    if args.k_base is not None:
+        cfg = cfg.with_(K_base=args.k_base)
     budget = cfg.budget if args.budget_mult is None else int(round(args.budget_mult * cfg.T))
+    budget = max(budget, cfg.K_base * cfg.T)
     return cfg, budget
 
 
@@ -258,7 +265,12 @@ def run_ours(args):
     shape = B.shape_of(cfg)
     layers = [synth.make_layer(cfg, l, device="cuda", with_x=(l == 0)) for l in range(n_layers)]
     if n_layers > 1:
-        budgets = [k * cfg.T for k in synth.stack_budgets(cfg)]
+        ks = synth.stack_budgets(cfg)
+        if args.stack_budgets == "alloc-l":
+            # Alloc-L (Sec. 3.2) on a seeded synthetic sensitivity matrix: the same total as the Dirichlet split
+            ks, _ = B.alloc_l_solve(synth.sensitivity_matrix(cfg), sum(ks))
+            ks = [max(k, cfg.K_base) for k in ks]
+        budgets = [k * cfg.T for k in ks]
     else:
         budgets = [budget]
     x0 = layers[0]["x"]

@@ -242,3 +242,19 @@ def score_rows(T: int, K_orig: int, key: int, ties: bool = False) -> torch.Tenso
     else:
         v = (s.to(torch.float32) + 1.0) / float(12 * 65535 + 2)
     return torch.sort(v, dim=1, descending=True).values.contiguous()
+
+
+def sensitivity_matrix(cfg: MoEConfig) -> List[List[float]]:
+    """A seeded stand-in for Alloc-L's profiled matrix S [L, K_orig] (the real one needs a trained model and a
+    calibration set): row i falls from a layer-specific level a_i at k = 1 to 0 at k = K_orig along (1 - (k-1)/(K-1))
+    to a layer-specific power in [1, 3], with a_i in [0.5, 1.5] larger for earlier layers on average, as the paper
+    reports for its profiles (earlier layers are more sensitive)."""
+    L, K = cfg.n_layers, cfg.K_orig
+    u = uniform01(2 * L, stream_key(cfg.seed, 0, _ID_BUDGET + 1))
+    rows = []
+    for i in range(L):
+        a = 0.5 + (1.0 - i / max(L - 1, 1)) * 0.6 + 0.4 * u[2 * i]
+        pw = 1.0 + 2.0 * u[2 * i + 1]
+        rows.append([a * (1.0 - (k - 1) / max(K - 1, 1)) ** pw for k in range(1, K + 1)])
+    return rows
+

@@ -62,3 +62,18 @@ def test_errors():
     with pytest.raises(B.MoeError) as ei:
         B.alloc_l_solve(np.full((2, 2), np.inf), 4)
     assert ei.value.status == B.MOE_ERR_NONFINITE
+
+
+def test_stack_budgets_from_the_synthetic_sensitivity_matrix():
+    """What `bench.py --stack-budgets alloc-l` runs: a decreasing, seeded S for the 26-layer stack, solved at the
+    same total (78) as the Dirichlet split; earlier layers are the more sensitive ones and get more on average."""
+    from paper_2604_08133_b200 import synth
+    cfg = synth.CONFIGS["c4"]
+    S = np.array(synth.sensitivity_matrix(cfg))
+    assert S.shape == (26, 6) and np.array_equal(S, np.array(synth.sensitivity_matrix(cfg)))
+    assert (np.diff(S, axis=1) <= 0).all() and (S[:, -1] == 0).all() and (S[:, 0] > 0).all()
+    ks, cost = B.alloc_l_solve(S, 78)
+    assert sum(ks) == 78 and all(1 <= k <= 6 for k in ks)
+    assert ks == orc.alloc_l_dp(S, 78)[0]
+    assert sum(ks[:13]) > sum(ks[13:])
+
