@@ -230,3 +230,16 @@ def test_other_model_shapes(name, T, mult):
     cfg = synth.CONFIGS[name].with_(T=T, budget=int(mult * T))
     _full_check(cfg)
 
+
+@pytest.mark.parametrize("T,H,N,I,S,K,kb,budget", [
+    (1, 64, 8, 64, 0, 2, 1, 1),            # one token, the smallest sizes the ABI accepts
+    (33, 192, 12, 128, 1, 3, 0, 40),        # N a multiple of 4 only, K_base 0, ragged everything
+    (130, 128, 128, 192, 0, 16, 2, 1000),   # the largest N and K_orig
+    (257, 256, 8, 64, 3, 4, 4, 1028),       # K_base = K_orig: nothing to redistribute, three shared experts
+    (300, 128, 8, 128, 2, 4, 1, 1200),      # budget = K_orig*T: plain Top-K_orig
+    (700, 128, 4 * 2, 256, 1, 2, 1, 1390),  # ~174 rows per expert: the CTA-pair tiles, with a shared expert
+])
+def test_odd_shapes(T, H, N, I, S, K, kb, budget):
+    cfg = synth.MoEConfig("odd", T=T, H=H, N=N, I=I, S=S, K_orig=K, K_base=kb, budget=budget, zipf_bias=(N >= 12), seed=T)
+    _full_check(cfg)
+
