@@ -233,12 +233,12 @@ static moe_status gate_launch_t(const moe_shape* s, const uint16_t* x, const uin
       return MOE_ERR_CUDA;
     attr_done = true;
   }
-  // CTAs per token tile: a power of two <= 8 that leaves every CTA at least one chunk, grown until
-  // the grid has about two CTAs per SM (more only adds cluster barriers)
+  // CTAs per token tile: a power of two <= 8 that leaves every CTA at least one chunk, grown while
+  // the grid stays within two CTAs per SM (measured: 256 CTAs beat 128 and 512 at 2048 and 4096 tokens)
   const int nchunks = (s->H + kGateKC - 1) / kGateKC;
   const int tiles = (s->T + TM - 1) / TM;
   int ks = 1;
-  while (ks * 2 <= 8 && ks * 2 <= nchunks && tiles * ks < 296) ks *= 2;
+  while (ks * 2 <= 8 && ks * 2 <= nchunks && tiles * ks * 2 <= 296) ks *= 2;
   const cudaError_t err = launch_dependent(
       moe_gate_kernel<NT16, NW>, dim3((unsigned)tiles, (unsigned)ks, 1), dim3(32 * NW), smem, stream, (unsigned)ks,
       reinterpret_cast<const __nv_bfloat16*>(x), reinterpret_cast<const __nv_bfloat16*>(W_gate), gate_bias, (int)s->T,
