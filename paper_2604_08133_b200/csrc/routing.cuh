@@ -17,6 +17,7 @@ struct SelectSmem {
   int scan_ws[33];
   uint32_t prefix;
   int remaining;
+  int bucket;
 };
 
 // The selection, run by one CTA of kSelThreads threads.  `smem_raw`: sizeof(SelectSmem) bytes, then
@@ -102,6 +103,7 @@ DEV void alloc_t_select_block(unsigned char* smem_raw, const float* __restrict__
           if (above < rem && rem <= above + c[q]) {
             sm.prefix = prefix | ((uint32_t)(255 - (lane * 8 + q)) << shift);
             sm.remaining = rem - above;
+            sm.bucket = c[q];            // keys that share the prefix chosen so far
             above = rem;                 // stop
           } else {
             above += c[q];
@@ -114,6 +116,21 @@ DEV void alloc_t_select_block(unsigned char* smem_raw, const float* __restrict__
   }
   const uint32_t tau = sm.prefix;
   const int need_eq = sm.remaining;       // how many keys equal to tau are kept (>= 1)
+
+  // After the last pass `bucket` is the number of keys equal to tau.  When all of them are kept (always
+  // the case when tau occurs once) no order among ties matters: one coalesced sweep over the tokens.
+  if (sm.bucket == need_eq) {
+    for (int t = tid; t < T; t += kSelThreads) {
+      int n = K_base;
+      for (int j = K_base; j < K_orig; ++j) {
+        const uint32_t k = use_smem_keys ? skeys[(long long)t * Kr + (j - K_base)] : bits[(long long)t * K_orig + j];
+        n += (k >= tau);
+      }
+      n_sel[t] = n;
+    }
+    __syncthreads();
+    return;
+  }
 
   // Per token: keys above tau, then ties in flat order.  Threads own contiguous token ranges.
   const int tpt = (T + kSelThreads - 1) / kSelThreads;
