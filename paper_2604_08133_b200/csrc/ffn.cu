@@ -15,9 +15,15 @@
 //
 // CTA = 6 warps: warp 0 lane 0 issues TMA loads (A 128x64, B 256x64 or 128x64 bf16, 128-byte
 // swizzle) into a ring of 4 (6) stages; warp 1 lane 0 issues tcgen05.mma (M=128, N=256 or 128,
-// K=16) into one of two TMEM accumulators; warps 2-5 read the finished accumulator with tcgen05.ld, apply
-// the epilogue and store bf16 rows (row-masked at the ragged end of an expert's run) while the
-// next tile's main loop runs.  Every mbarrier wait is bounded (see common.cuh).
+// K=16) into one of two TMEM accumulators; warps 2-5 read the finished accumulator with
+// tcgen05.ld, apply the epilogue and store bf16 rows (row-masked at the ragged end of an expert's
+// run) while the next tile's main loop runs.  Every wait is bounded (see common.cuh).
+//
+// Two variants of the kernel: one CTA per 128-row tile (ffn_gemm_kernel) and a CTA pair per 256-row
+// tile (ffn_gemm_pair_kernel, tcgen05 cta_group::2); launch_ffn picks by shape.  GEMM-2 is launched
+// as a programmatic dependent that does not wait for the whole of GEMM-1: per block of token rows
+// GEMM-1's epilogue counts finished tiles of h and GEMM-2's producer loads a block once its count is
+// complete, so GEMM-2 fills the SMs that GEMM-1's last round of tiles leaves idle.
 #include <cuda.h>
 #include <stdlib.h>
 
