@@ -166,6 +166,10 @@ CONFIGS: Dict[str, MoEConfig] = {
     # 2-3.5 per token) and OLMoE-shaped (64 routed experts, Top-8, budgets 4-7).  The paper gives the expert counts
     # and Top-K only; hidden and intermediate sizes and the shared expert are synthetic choices.
     "qwen": MoEConfig("qwen", T=4096, H=2048, N=60, I=1408, S=1, K_orig=4, K_base=1, budget=int(2.5 * 4096)),
+    # the batch shapes of the paper's own timing run (App. A.2: batch 8; decode = 8 tokens per step, prefill = 8
+    # prompts of 32 tokens) on the DeepSeek-V2-Lite-shaped layer, at half budget
+    "d8": MoEConfig("d8", T=8, H=2048, N=64, I=1408, S=2, K_orig=6, K_base=1, budget=24, zipf_bias=True),
+    "p256": MoEConfig("p256", T=256, H=2048, N=64, I=1408, S=2, K_orig=6, K_base=1, budget=768, zipf_bias=True),
     "olmoe": MoEConfig("olmoe", T=4096, H=2048, N=64, I=1024, S=0, K_orig=8, K_base=1, budget=5 * 4096),
 }
 
