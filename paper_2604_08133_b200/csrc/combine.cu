@@ -26,29 +26,42 @@ combine_kernel(const uint4* __restrict__ y_perm, const int32_t* __restrict__ pai
   const int t = blockIdx.x;
   pdl_prologue_done();
   if (threadIdx.x < 16) {
+    // the count, the position and the weight of column j do not depend on each other: one round trip
     const int j = threadIdx.x;
-    const int n = min(max(n_sel[t], 0), K_orig);
-    if (j == 0) s_n = n;
+    const int n = min(max(__ldg(n_sel + t), 0), K_orig);
     int pos = -1;
     float w = 0.f;
-    if (j < n) {
-      pos = pair_pos[(long long)t * K_orig + j];
-      w = topk_score[(long long)t * K_orig + j];
-      if (pos < 0 || pos >= budget_rows) { pos = -1; w = 0.f; }
+    if (j < K_orig) {
+      pos = __ldg(pair_pos + (long long)t * K_orig + j);
+      w = __ldg(topk_score + (long long)t * K_orig + j);
     }
+    if (j >= n || pos < 0 || pos >= budget_rows) { pos = -1; w = 0.f; }
+    if (j == 0) s_n = n;
     s_pos[j] = pos;
     s_w[j] = w;
   }
   __syncthreads();
   const int n = s_n;
   for (int c = threadIdx.x; c < row_vec; c += blockDim.x) {
+    // the token's own rows first, then the expert rows four loads at a time, FMAs in ascending j
+    uint4 vs = make_uint4(0, 0, 0, 0), vr = make_uint4(0, 0, 0, 0);
+    if (y_shared != nullptr) vs = __ldg(y_shared + (long long)t * row_vec + c);
+    if (x_res != nullptr) vr = __ldg(x_res + (long long)t * row_vec + c);
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    for (int j = 0; j < n; ++j) {
-      const int pos = s_pos[j];
-      if (pos >= 0) fma8(acc, __ldg(y_perm + (long long)pos * row_vec + c), s_w[j]);
+    for (int jb = 0; jb < n; jb += 4) {
+      uint4 v[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int pos = s_pos[jb + q < 16 ? jb + q : 15];
+        v[q] = make_uint4(0, 0, 0, 0);
+        if (jb + q < n && pos >= 0) v[q] = __ldg(y_perm + (long long)pos * row_vec + c);
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (jb + q < n) fma8(acc, v[q], s_w[jb + q < 16 ? jb + q : 15]);
     }
-    if (y_shared != nullptr) fma8(acc, __ldg(y_shared + (long long)t * row_vec + c), 1.f);
-    if (x_res != nullptr) fma8(acc, __ldg(x_res + (long long)t * row_vec + c), 1.f);
+    if (y_shared != nullptr) fma8(acc, vs, 1.f);
+    if (x_res != nullptr) fma8(acc, vr, 1.f);
     uint4 o;
     o.x = pack_bf16x2(acc[0], acc[1]);
     o.y = pack_bf16x2(acc[2], acc[3]);
