@@ -167,12 +167,15 @@ DEV void build_masks(uint32_t* mask, const int32_t* __restrict__ topk_idx, const
   __syncwarp();
   n_out = 0;
   if (t < T) {
-    n_out = min(max(n_sel[t], 0), K_orig);
+    // the count and all K_orig expert ids travel together (one round trip); ids past the count are ignored
+    const int n_raw = n_sel[t];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) e_out[j] = (j < K_orig) ? topk_idx[(long long)t * K_orig + j] : 0;
+    n_out = min(max(n_raw, 0), K_orig);
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
       if (j < n_out) {
-        int e = topk_idx[(long long)t * K_orig + j];
-        e = min(max(e, 0), N - 1);   // keeps every access in bounds on corrupt input
+        const int e = min(max(e_out[j], 0), N - 1);   // keeps every access in bounds on corrupt input
         e_out[j] = e;
         atomicOr(&mask[e], 1u << lane);
       }
@@ -224,23 +227,28 @@ DEV void permute_place_warp(uint32_t* mask, const int32_t* __restrict__ topk_idx
   build_masks(mask, topk_idx, n_sel, t, T, N, K_orig, lane, e_loc, n);
   if (t >= T) return;
   const uint32_t lower = (1u << lane) - 1u;
+  float w[16];   // all of the token's scores in one round trip
+#pragma unroll
+  for (int j = 0; j < 16; ++j) w[j] = (j < K_orig) ? topk_score[(long long)t * K_orig + j] : 0.f;
+  int pos[16];
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
-    if (j < K_orig) {
-      int pos = -1;
-      if (j < n) {
-        const int e = e_loc[j];
-        pos = seg_base[(long long)e * nseg + seg] + __popc(mask[e] & lower);
-        if (pos >= 0 && pos < budget) {   // always true when sum n_sel == budget
-          perm_token[pos] = t;
-          perm_weight[pos] = topk_score[(long long)t * K_orig + j];
-        } else {
-          pos = -1;
-        }
-      }
-      pair_pos[(long long)t * K_orig + j] = pos;
+    pos[j] = -1;
+    if (j < n) {
+      const int e = e_loc[j];
+      const int q = seg_base[(long long)e * nseg + seg] + __popc(mask[e] & lower);
+      if (q >= 0 && q < budget) pos[j] = q;   // always true when sum n_sel == budget
     }
   }
+#pragma unroll
+  for (int j = 0; j < 16; ++j)
+    if (j < K_orig && pos[j] >= 0) {
+      perm_token[pos[j]] = t;
+      perm_weight[pos[j]] = w[j];
+    }
+#pragma unroll
+  for (int j = 0; j < 16; ++j)
+    if (j < K_orig) pair_pos[(long long)t * K_orig + j] = pos[j];
 }
 
 }  // namespace allocmoe
