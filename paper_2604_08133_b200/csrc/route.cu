@@ -31,15 +31,22 @@ moe_route_kernel(const float* __restrict__ topk_score, const int32_t* __restrict
   alloc_t_select_block(smem_raw, topk_score, T, K_orig, K_base, budget - (long long)K_base * T, use_smem_keys, n_sel,
                        dev_status);   // ends with a block barrier: n_sel is visible, the pool is free
 
+  // Every warp owns at most one 32-token segment here (moe_route_fits), so the masks and expert ids
+  // built for the count are still there for the placement: nothing is loaded twice.
   uint32_t* mask = reinterpret_cast<uint32_t*>(sm.warp_hist[warp]);
-  for (int seg = warp; seg < nseg; seg += kRouteWarps)
-    permute_count_warp(mask, topk_idx, n_sel, seg, T, N, K_orig, nseg, seg_counts);
+  const int lane = threadIdx.x & 31;
+  const int seg = warp;
+  int e_loc[16], n = 0;
+  if (seg < nseg) {
+    build_masks(mask, topk_idx, n_sel, seg * 32 + lane, T, N, K_orig, lane, e_loc, n);
+    for (int e = lane; e < N; e += 32) seg_counts[(long long)e * nseg + seg] = __popc(mask[e]);
+  }
   __syncthreads();
   permute_scan_block(seg_counts, N, nseg, budget, expert_offsets, dev_status, sm.scan_ws);
   __syncthreads();
-  for (int seg = warp; seg < nseg; seg += kRouteWarps)
-    permute_place_warp(mask, topk_idx, topk_score, n_sel, seg, T, N, K_orig, nseg, seg_counts, budget, perm_token,
-                       perm_weight, pair_pos);
+  if (seg < nseg)
+    permute_place_from_masks(mask, e_loc, n, topk_score, seg, T, K_orig, nseg, seg_counts, budget, perm_token,
+                             perm_weight, pair_pos);
 }
 
 }  // namespace allocmoe

@@ -216,15 +216,30 @@ DEV void permute_scan_block(int32_t* seg_counts, int N, int nseg, long long budg
   }
 }
 
+DEV void permute_place_from_masks(const uint32_t* mask, const int (&e_loc)[16], int n,
+                                  const float* __restrict__ topk_score, int seg, int T, int K_orig, int nseg,
+                                  const int32_t* seg_base, long long budget, int32_t* __restrict__ perm_token,
+                                  float* __restrict__ perm_weight, int32_t* __restrict__ pair_pos);
+
 // One warp, one 32-token segment: list positions of its kept pairs.
 DEV void permute_place_warp(uint32_t* mask, const int32_t* __restrict__ topk_idx, const float* __restrict__ topk_score,
                             const int32_t* __restrict__ n_sel, int seg, int T, int N, int K_orig, int nseg,
                             const int32_t* seg_base, long long budget, int32_t* __restrict__ perm_token,
                             float* __restrict__ perm_weight, int32_t* __restrict__ pair_pos) {
   const int lane = threadIdx.x & 31;
-  const int t = seg * 32 + lane;
   int e_loc[16], n;
-  build_masks(mask, topk_idx, n_sel, t, T, N, K_orig, lane, e_loc, n);
+  build_masks(mask, topk_idx, n_sel, seg * 32 + lane, T, N, K_orig, lane, e_loc, n);
+  permute_place_from_masks(mask, e_loc, n, topk_score, seg, T, K_orig, nseg, seg_base, budget, perm_token, perm_weight,
+                           pair_pos);
+}
+
+// The placement proper, from the segment's masks and this lane's expert ids (build_masks).
+DEV void permute_place_from_masks(const uint32_t* mask, const int (&e_loc)[16], int n,
+                                  const float* __restrict__ topk_score, int seg, int T, int K_orig, int nseg,
+                                  const int32_t* seg_base, long long budget, int32_t* __restrict__ perm_token,
+                                  float* __restrict__ perm_weight, int32_t* __restrict__ pair_pos) {
+  const int lane = threadIdx.x & 31;
+  const int t = seg * 32 + lane;
   if (t >= T) return;
   const uint32_t lower = (1u << lane) - 1u;
   float w[16];   // all of the token's scores in one round trip
