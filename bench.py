@@ -32,10 +32,16 @@ NCU_TRAFFIC_BYTES = {
 }
 
 
-def kernels_per_layer(T):
+GATHER_ROWS_PER_EXPERT = 32     # the library's default: up to this many rows per routed expert GEMM-1 reads x by index
+
+
+def kernels_per_layer(cfg, budget):
     """Launches of one moe_layer_forward call: gate, routing (one fused launch up to 1024 tokens, else
-    select + permute count/scan/place), row gather, 2 expert GEMMs, combine."""
-    return 6 if T <= 1024 else 9
+    select + permute count/scan/place), row gather (none where the expert GEMM fetches the rows of x
+    itself), 2 expert GEMMs, combine."""
+    routing = 1 if cfg.T <= 1024 else 4
+    gather = 0 if budget <= GATHER_ROWS_PER_EXPERT * cfg.N else 1
+    return 1 + routing + gather + 2 + 1
 
 
 def parse_args():
@@ -335,7 +341,7 @@ def run_ours(args):
                    "layers": n_layers, "parallelism": "independent batches per GPU, replicated weights, no collective",
                    "l2": "weights exceed L2 (no flush)" if (cfg.N + cfg.S) * 6 * cfg.H * cfg.I > 126e6 else
                          "L2-resident workload, no flush (latency-bound case)"},
-        "clocks": clocks, "gpu_launches": (kernels_per_layer(cfg.T) + (1 if stack else 0)) * n_layers * steps,
+        "clocks": clocks, "gpu_launches": sum(kernels_per_layer(cfg, b) + (1 if stack else 0) for b in budgets) * steps,
     }
 
     peaks = load_peaks()

@@ -14,10 +14,11 @@ moe_status launch_gather_rows(const moe_shape*, const uint16_t*, const int32_t*,
 bool moe_route_fits(const moe_shape*);
 moe_status launch_moe_route(const moe_shape*, const float*, const int32_t*, int64_t, int32_t*, int32_t*, int32_t*, float*,
                             int32_t*, int32_t*, cudaStream_t);
-moe_status launch_ffn(const moe_shape*, const uint16_t*, const int32_t*, int64_t, const uint16_t*, const uint16_t*,
+moe_status launch_ffn(const moe_shape*, const uint16_t*, const int32_t*, const int32_t*, int64_t, const uint16_t*, const uint16_t*,
                       uint16_t*, uint16_t*, const uint16_t*, const uint16_t*, const uint16_t*, uint16_t*, uint16_t*,
                       int32_t*, int32_t*, cudaStream_t, cudaEvent_t);
 size_t ffn_done_ints(const moe_shape*, int64_t);
+bool ffn_gathers(const moe_shape*, int64_t);
 moe_status launch_moe_combine(const moe_shape*, const uint16_t*, const int32_t*, const float*, const int32_t*,
                               const uint16_t*, const uint16_t*, long long, uint16_t*, cudaStream_t);
 moe_status launch_rmsnorm(const moe_shape*, const uint16_t*, uint16_t*, cudaStream_t);
@@ -161,7 +162,7 @@ moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_perm, const
   if (budget < 0 || budget > (int64_t)shape->K_orig * shape->T) return MOE_ERR_BUDGET;
   const WsLayout L = ws_layout(shape, budget);
   if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
-  return launch_ffn(shape, x_perm, expert_offsets, budget, W13, W2, at<uint16_t>(ws, L.h), y_perm, nullptr, nullptr,
+  return launch_ffn(shape, x_perm, nullptr, expert_offsets, budget, W13, W2, at<uint16_t>(ws, L.h), y_perm, nullptr, nullptr,
                     nullptr, nullptr, nullptr, dev_status, at<int32_t>(ws, L.gemm_done), (cudaStream_t)stream, nullptr);
 }
 
@@ -171,7 +172,7 @@ moe_status moe_shared_ffn(const moe_shape* shape, const uint16_t* x, const uint1
   if (!aligned16(x) || !aligned16(Wsh13) || !aligned16(Wsh2) || !aligned16(y_shared) || !aligned16(ws)) return MOE_ERR_ARG;
   const WsLayout L = ws_layout(shape, 0);
   if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
-  return launch_ffn(shape, nullptr, nullptr, 0, nullptr, nullptr, nullptr, nullptr, x, Wsh13, Wsh2,
+  return launch_ffn(shape, nullptr, nullptr, nullptr, 0, nullptr, nullptr, nullptr, nullptr, x, Wsh13, Wsh2,
                     at<uint16_t>(ws, L.h_sh), y_shared, dev_status, at<int32_t>(ws, L.gemm_done), (cudaStream_t)stream,
                     nullptr);
 }
@@ -210,6 +211,9 @@ moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const ui
   uint16_t* y_perm = at<uint16_t>(ws, L.y_perm);
   uint16_t* y_shared = shape->S > 0 ? at<uint16_t>(ws, L.y_shared) : nullptr;
 
+  // for short expert runs GEMM-1 fetches the routed tokens' rows from x by index and no permuted copy is made
+  if (ffn_gathers(shape, budget)) x_perm = nullptr;
+
   prof_mark(0, st);
   moe_status r = launch_moe_gate(shape, x, W_gate, gate_bias, nullptr, topk_idx, topk_score, st);
   if (r != MOE_OK) return r;
@@ -220,7 +224,7 @@ moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const ui
                          dev_status, st);
     if (r != MOE_OK) return r;
     prof_mark(2, st);
-    if (budget > 0) r = launch_gather_rows(shape, x, perm_token, budget, x_perm, st);
+    if (budget > 0 && x_perm != nullptr) r = launch_gather_rows(shape, x, perm_token, budget, x_perm, st);
   } else {
     r = launch_alloc_t_select(shape, topk_score, budget, n_sel, dev_status, st);
     if (r != MOE_OK) return r;
@@ -230,7 +234,8 @@ moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const ui
   }
   if (r != MOE_OK) return r;
   prof_mark(3, st);
-  r = launch_ffn(shape, x_perm, expert_offsets, budget, W13, W2, at<uint16_t>(ws, L.h), y_perm,
+  r = launch_ffn(shape, x_perm != nullptr ? x_perm : x, x_perm != nullptr ? nullptr : perm_token, expert_offsets, budget,
+                 W13, W2, at<uint16_t>(ws, L.h), y_perm,
                  shape->S > 0 ? x : nullptr, Wsh13, Wsh2, at<uint16_t>(ws, L.h_sh), y_shared, dev_status,
                  at<int32_t>(ws, L.gemm_done), st, g_prof_on ? g_prof_ev[4] : nullptr);
   if (r != MOE_OK) return r;

@@ -179,6 +179,16 @@ DEV void tma_load_3d(void* smem_dst, const void* tmap, uint64_t* bar, int c0, in
       : "memory");
 }
 
+// Four rows of a 2-D tensor picked by row index (the map's box is 64 columns x 1 row): 4 x 128 bytes,
+// stored as four consecutive rows of the 128-byte-swizzled tile that smem_dst lies in.
+DEV void tma_gather4_2d(void* smem_dst, const void* tmap, uint64_t* bar, int c0, int r0, int r1, int r2, int r3) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"((uint64_t)tmap), "r"(smem_u32(bar)), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
+      : "memory");
+}
+
 // ------------------------------------------------------------------ tcgen05 / TMEM
 DEV void tmem_alloc(uint32_t* smem_result, uint32_t ncols) {   // whole warp
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)), "r"(ncols) : "memory");
@@ -269,6 +279,14 @@ DEV void tma_load_3d_pair(void* smem_dst, const void* tmap, uint32_t bar_cluster
   asm volatile(
       "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_u32(smem_dst)), "l"((uint64_t)tmap), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+DEV void tma_gather4_2d_pair(void* smem_dst, const void* tmap, uint32_t bar_cluster_addr, int c0, int r0, int r1, int r2,
+                             int r3) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes.cta_group::2"
+      " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"((uint64_t)tmap), "r"(bar_cluster_addr), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
       : "memory");
 }
 DEV void tmem_alloc_pair(uint32_t* smem_result, uint32_t ncols) {   // the same warp of both CTAs

@@ -66,7 +66,40 @@ struct FfnGemmParams {
   // the count reaches dep_need_* (GEMM-1's tiles per block x epilogue warps).  nullptr = no tracking.
   int32_t* done;
   int dep_need_routed, dep_need_shared;
+  // gather_rows > 0: the routed A tensor map has a box one row high and the producer warp fetches a
+  // tile's rows four per TMA instruction, only those that hold rows of the expert's run.  GEMM-1 can
+  // then read the routed tokens' rows straight from x instead of a permuted copy: row m of the routed
+  // A matrix is x[gather_idx[m]] (gather_idx = perm_token, gather_rows entries); with gather_idx ==
+  // nullptr row m is row m (GEMM-2 on h).  gather_rows == 0: A rows come as one 128-row box.
+  const int32_t* gather_idx;
+  int gather_rows;
 };
+
+// Token rows a producer lane fetches per stage when A is gathered: lane l owns rows 4l..4l+3 of the tile.
+struct GatherRows {
+  int r[4];
+  bool issue;          // this lane's four rows hold at least one row of the expert's run
+  uint32_t a_bytes;    // bytes of A all lanes together bring in per stage
+};
+// Rows past the end of the run inside a fetched group of four take the index of the list's last valid
+// entry; groups wholly past the end are not fetched at all (their rows of the accumulator are never
+// stored), which at decode sizes leaves half a KB of A per stage instead of 16 KB.
+DEV GatherRows gather_rows_of_tile(const FfnGemmParams& p, int a_row, int m_end, int lane, int tile_rows) {
+  GatherRows g;
+  const int valid = min(max(m_end - a_row, 0), tile_rows);
+  g.issue = 4 * lane < valid;
+  g.a_bytes = (uint32_t)((valid + 3) / 4) * 512u;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) g.r[i] = 0;
+  if (g.issue) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int m = min(a_row + 4 * lane + i, p.gather_rows - 1);
+      g.r[i] = p.gather_idx != nullptr ? __ldg(p.gather_idx + m) : m;
+    }
+  }
+  return g;
+}
 
 struct FfnSmemCtl {
   uint64_t full[kMaxStages];
@@ -189,7 +222,10 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
 
   if (warp == 0) {
     // ======================= TMA producer =======================
-    if (lane == 0) {
+    // Lane 0 issues the box loads.  With gathered A rows (FfnGemmParams::gather_rows) the whole warp runs
+    // the loop and every lane fetches its four rows of a routed tile per stage.
+    const bool gather = p.gather_rows > 0;
+    if (lane == 0 || gather) {
       TileWalker<kSwiGLU, kN, kBM> w(ctl, p);
       uint32_t it = 0;
       bool ok = true;
@@ -204,34 +240,52 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
           if (kSwiGLU) { e_n = tc.nb / w.nb_routed; n_row = (tc.nb % w.nb_routed) * kOutCols; }
           else { e_n = 0; }
         }
+        const bool gtile = gather && !tc.shared;
+        GatherRows gr{};
+        if (gtile) gr = gather_rows_of_tile(p, tc.m0, tc.m_end, lane, kBM);
         if (!kSwiGLU && p.done != nullptr) {   // the block's rows of h are complete?
-          if (!(ok = flag_wait_bounded(p.done + tc.dep_id, tc.shared ? p.dep_need_shared : p.dep_need_routed,
-                                       abort_flag, p.dev_status)))
-            break;
+          if (lane == 0)
+            ok = flag_wait_bounded(p.done + tc.dep_id, tc.shared ? p.dep_need_shared : p.dep_need_routed, abort_flag,
+                                   p.dev_status);
+          if (gather) {
+            __syncwarp();
+            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+          }
+          if (!ok) break;
           fence_proxy_async_global();
         }
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!(ok = mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status))) break;
+          ok = gather ? mbar_wait_bounded_warp(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status)
+                      : mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status);
+          if (!ok) break;
           unsigned char* sa = tiles + s * kStageBytes;
           unsigned char* sb = sa + kABytes;
-          mbar_expect_tx(&ctl->full[s], kStageBytes);
-          tma_load_2d(sa, tmA, &ctl->full[s], kb * kBK, tc.m0);
-          int e_k = e_n, k_col = kb * kBK;
-          if (tc.shared && !kSwiGLU) { e_k = kb / kb_routed; k_col = (kb % kb_routed) * kBK; }
-          if (kSwiGLU) {
-            tma_load_3d(sb, tmB, &ctl->full[s], k_col, n_row, e_k);
-            tma_load_3d(sb + kBBytes / 2, tmB, &ctl->full[s], k_col, p.up_row_offset + n_row, e_k);
-          } else {
-            tma_load_3d(sb, tmB, &ctl->full[s], k_col, n_row, e_k);
+          if (lane == 0) {
+            mbar_expect_tx(&ctl->full[s], gtile ? gr.a_bytes + kBBytes : kStageBytes);
+            if (!gtile) tma_load_2d(sa, tmA, &ctl->full[s], kb * kBK, tc.m0);
+            int e_k = e_n, k_col = kb * kBK;
+            if (tc.shared && !kSwiGLU) { e_k = kb / kb_routed; k_col = (kb % kb_routed) * kBK; }
+            if (kSwiGLU) {
+              tma_load_3d(sb, tmB, &ctl->full[s], k_col, n_row, e_k);
+              tma_load_3d(sb + kBBytes / 2, tmB, &ctl->full[s], k_col, p.up_row_offset + n_row, e_k);
+            } else {
+              tma_load_3d(sb, tmB, &ctl->full[s], k_col, n_row, e_k);
+            }
+          }
+          if (gtile) {
+            __syncwarp();   // the stage's byte count is announced before any lane's rows can land
+            if (gr.issue) tma_gather4_2d(sa + lane * 512, tmA, &ctl->full[s], kb * kBK, gr.r[0], gr.r[1], gr.r[2], gr.r[3]);
           }
         }
       }
-      // drain: every load this thread issued must have landed before the CTA may exit
-      const uint32_t issued = it;
-      for (uint32_t q = (issued > (uint32_t)kStages ? issued - kStages : 0u); q < issued; ++q)
-        mbar_wait_drain(&ctl->full[q % kStages], (q / kStages) & 1u);
+      // drain: every load this warp issued must have landed before the CTA may exit
+      if (lane == 0) {
+        const uint32_t issued = it;
+        for (uint32_t q = (issued > (uint32_t)kStages ? issued - kStages : 0u); q < issued; ++q)
+          mbar_wait_drain(&ctl->full[q % kStages], (q / kStages) & 1u);
+      }
     }
   } else if (warp == 1) {
     // ======================= MMA issuer =======================
@@ -445,7 +499,8 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
 
   if (warp == 0) {
     // ======================= TMA producer (both CTAs) =======================
-    if (lane == 0) {
+    const bool gather = p.gather_rows > 0;   // see the one-CTA kernel
+    if (lane == 0 || gather) {
       TileWalker<kSwiGLU, kN, kPairM> w(ctl, p);
       uint32_t it = 0;
       bool ok = true;
@@ -462,35 +517,53 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
         // this CTA's half of the B tile: GEMM-1 W1 rows (leader) or W3 rows (peer); GEMM-2 rows +128*rank
         const int b_row = kSwiGLU ? (rank == 0 ? n_row : p.up_row_offset + n_row) : n_row + (int)rank * (kN / 2);
         const int a_row = tc.m0 + (int)rank * kBM;
+        const bool gtile = gather && !tc.shared;
+        GatherRows gr{};
+        if (gtile) gr = gather_rows_of_tile(p, a_row, tc.m_end, lane, kBM);
         if (!kSwiGLU && p.done != nullptr) {   // the block's rows of h are complete?
-          if (!(ok = flag_wait_bounded(p.done + tc.dep_id, tc.shared ? p.dep_need_shared : p.dep_need_routed,
-                                       abort_flag, p.dev_status)))
-            break;
+          if (lane == 0)
+            ok = flag_wait_bounded(p.done + tc.dep_id, tc.shared ? p.dep_need_shared : p.dep_need_routed, abort_flag,
+                                   p.dev_status);
+          if (gather) {
+            __syncwarp();
+            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+          }
+          if (!ok) break;
           fence_proxy_async_global();
         }
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % kPairStages;
           const uint32_t ph = (it / kPairStages) & 1u;
-          if (!(ok = mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status))) break;
+          ok = gather ? mbar_wait_bounded_warp(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status)
+                      : mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status);
+          if (!ok) break;
           unsigned char* sa = tiles + s * kPairStageBytes;
           unsigned char* sb = sa + kABytes;
           const uint32_t bar = cluster_addr_of(&ctl->full[s], 0);
-          mbar_expect_tx_cluster(bar, kPairStageBytes);
-          tma_load_2d_pair(sa, tmA, bar, kb * kBK, a_row);
-          int e_k = e_n, k_col = kb * kBK;
-          if (tc.shared && !kSwiGLU) { e_k = kb / kb_routed; k_col = (kb % kb_routed) * kBK; }
-          tma_load_3d_pair(sb, tmB, bar, k_col, b_row, e_k);
+          if (lane == 0) {
+            mbar_expect_tx_cluster(bar, gtile ? gr.a_bytes + kABytes : kPairStageBytes);
+            if (!gtile) tma_load_2d_pair(sa, tmA, bar, kb * kBK, a_row);
+            int e_k = e_n, k_col = kb * kBK;
+            if (tc.shared && !kSwiGLU) { e_k = kb / kb_routed; k_col = (kb % kb_routed) * kBK; }
+            tma_load_3d_pair(sb, tmB, bar, k_col, b_row, e_k);
+          }
+          if (gtile) {
+            __syncwarp();   // the stage's byte count is announced before any lane's rows can land
+            if (gr.issue) tma_gather4_2d_pair(sa + lane * 512, tmA, bar, kb * kBK, gr.r[0], gr.r[1], gr.r[2], gr.r[3]);
+          }
         }
       }
       // drain: the last loads have landed once the leader's barriers of the last stages completed;
       // the peer learns it through the multicast `empty` that follows.  Wait for what was issued.
-      const uint32_t issued = it;
-      if (rank == 0) {
-        for (uint32_t q = (issued > (uint32_t)kPairStages ? issued - kPairStages : 0u); q < issued; ++q)
-          mbar_wait_drain(&ctl->full[q % kPairStages], (q / kPairStages) & 1u);
-      } else {
-        for (uint32_t q = (issued > (uint32_t)kPairStages ? issued - kPairStages : 0u); q < issued; ++q)
-          mbar_wait_drain(&ctl->empty[q % kPairStages], (q / kPairStages) & 1u);
+      if (lane == 0) {
+        const uint32_t issued = it;
+        if (rank == 0) {
+          for (uint32_t q = (issued > (uint32_t)kPairStages ? issued - kPairStages : 0u); q < issued; ++q)
+            mbar_wait_drain(&ctl->full[q % kPairStages], (q / kPairStages) & 1u);
+        } else {
+          for (uint32_t q = (issued > (uint32_t)kPairStages ? issued - kPairStages : 0u); q < issued; ++q)
+            mbar_wait_drain(&ctl->empty[q % kPairStages], (q / kPairStages) & 1u);
+        }
       }
     }
   } else if (warp == 1) {
@@ -735,9 +808,27 @@ size_t ffn_done_ints(const moe_shape* s, int64_t budget) {
   return (size_t)(budget / kBM + s->N + (s->S > 0 ? s->T / kBM + 1 : 0) + 4);
 }
 
+// Fetching A rows four per TMA instruction costs the producer one instruction per four rows and
+// stage where a box load costs one per stage: measured, it pays while an expert's run is short (the
+// weight stream leaves the TMA unit idle and most of a 128-row box would be padding) and loses
+// badly on full tiles (prefill step 0.46 -> 0.72 ms).  Used up to ALLOCMOE_GATHER (default 32) rows
+// per routed expert on average; 0 = never.
+bool ffn_gathers(const moe_shape* s, int64_t budget) {
+  static int limit = -1;
+  if (limit < 0) {
+    limit = 32;
+    const char* e = getenv("ALLOCMOE_GATHER");
+    if (e != nullptr && atoi(e) >= 0) limit = atoi(e);
+  }
+  return budget > 0 && budget <= (int64_t)limit * s->N;
+}
+
 // Routed and/or shared experts in one pair of launches.
 //   routed part present iff budget > 0 && x_perm != nullptr; shared part iff S > 0 && x_shared != nullptr.
-moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t* expert_offsets, int64_t budget,
+//   gather_idx != nullptr: x_perm is x [T, H] itself and routed row m is x[gather_idx[m]] (perm_token);
+//   callers pass it only where ffn_gathers() holds.
+moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t* gather_idx,
+                      const int32_t* expert_offsets, int64_t budget,
                       const uint16_t* W13, const uint16_t* W2, uint16_t* h, uint16_t* y_perm, const uint16_t* x_shared,
                       const uint16_t* Wsh13, const uint16_t* Wsh2, uint16_t* h_sh, uint16_t* y_shared,
                       int32_t* dev_status, int32_t* done, cudaStream_t stream, cudaEvent_t between) {
@@ -750,11 +841,13 @@ moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t*
   const int tile_n = pairs ? 256 : pick_tile_n(s, routed ? budget : 0, shared);
   const uint32_t kUmmaN = (uint32_t)tile_n;
   const uint32_t b2_box = pairs ? kUmmaN / 2 : kUmmaN;   // a pair's CTA loads half of the B tile
+  const bool by_rows = routed && (gather_idx != nullptr || ffn_gathers(s, budget));
   bool ok = true;
   if (routed) {
-    ok &= make_tmap(&a1r, x_perm, H, (uint64_t)budget, 0, H, 0, kBM);
+    if (gather_idx != nullptr) ok &= make_tmap(&a1r, x_perm, H, (uint64_t)s->T, 0, H, 0, 1);
+    else ok &= make_tmap(&a1r, x_perm, H, (uint64_t)budget, 0, H, 0, by_rows ? 1 : kBM);
     ok &= make_tmap(&b1r, W13, H, 2 * I, (uint64_t)s->N, H, 2 * I * H, kUmmaN / 2);
-    ok &= make_tmap(&a2r, h, I, (uint64_t)budget, 0, I, 0, kBM);
+    ok &= make_tmap(&a2r, h, I, (uint64_t)budget, 0, I, 0, by_rows ? 1 : kBM);
     ok &= make_tmap(&b2r, W2, I, H, (uint64_t)s->N, I, H * I, b2_box);
   }
   if (shared) {
@@ -785,6 +878,8 @@ moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t*
       return MOE_ERR_CUDA;
   }
   // GEMM-1
+  p.gather_idx = routed ? gather_idx : nullptr;
+  p.gather_rows = by_rows ? (int)budget : 0;
   p.n_per_sub = s->I;
   p.k_per_sub = s->H;
   p.up_row_offset = s->I;
@@ -798,6 +893,8 @@ moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t*
   if (st != MOE_OK) return st;
   if (between != nullptr) cudaEventRecord(between, stream);
   // GEMM-2
+  p.gather_idx = nullptr;
+  p.gather_rows = by_rows ? (int)budget : 0;
   p.n_per_sub = s->H;
   p.k_per_sub = s->I;
   p.up_row_offset = 0;

@@ -284,18 +284,21 @@ def test_combine_against_oracle_formula():
     assert max_rel(got, want) <= 4e-3
 
 
-@pytest.mark.parametrize("pair", ["0", "1"])
-def test_expert_gemm_variants_forced(pair):
-    """The library picks one-CTA or CTA-pair tiles by shape; both must be right on every shape.  The choice is read
-    from the environment once per process, so each forced setting runs the expert-GEMM tests in a process of its own."""
+@pytest.mark.parametrize("pair,gather", [("0", "0"), ("1", "0"), ("0", "1000000"), ("1", "1000000")])
+def test_expert_gemm_variants_forced(pair, gather):
+    """The library picks one-CTA or CTA-pair tiles, and box loads or row-by-row fetches of the token rows (from a
+    permuted copy or straight from x through perm_token), by shape; every combination must be right on every shape.
+    The choices are read from the environment once per process, so each forced setting runs the expert-GEMM tests and
+    the small whole-layer tests in a process of its own."""
     import os
     import subprocess
     import sys
     if os.environ.get("ALLOCMOE_PAIR") is not None:
         pytest.skip("already inside a forced run")
-    env = dict(os.environ, ALLOCMOE_PAIR=pair)
+    env = dict(os.environ, ALLOCMOE_PAIR=pair, ALLOCMOE_GATHER=gather)
     here = os.path.dirname(os.path.abspath(__file__))
-    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(here, "test_gpu_steps.py"), "-m", "gpu", "-q", "-x",
-                        "-k", "grouped_ffn or shared_ffn"], env=env, capture_output=True, text=True, timeout=600)
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(here, "test_gpu_steps.py"),
+                        os.path.join(here, "test_gpu_layer.py"), "-m", "gpu", "-q", "-x", "-k",
+                        "grouped_ffn or shared_ffn or c1_ or c2_decode or ragged_multi_tile or other_model_shapes "
+                        "or odd_shapes"], env=env, capture_output=True, text=True, timeout=900)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
-
