@@ -7,11 +7,11 @@
 // Both are C = A B^T with A [rows, K] and B [n, K] K-contiguous, i.e. both operands K-major.
 //
 // One persistent kernel per GEMM: grid = number of SMs, every CTA walks the tile list
-// tile = blockIdx.x, += gridDim.x.  The list is built on the device from expert_offsets (row
-// counts are data dependent): groups in order, inside a group column blocks outermost and
+// tile = blockIdx.x, += gridDim.x (TileSched).  The list is built on the device from expert_offsets
+// (row counts are data dependent): groups in order, inside a group column blocks outermost and
 // 128-row blocks innermost, so CTAs that run concurrently share a weight tile through L2.
-// A "group" is a routed expert or, last, the shared experts (all T rows; their S sub-experts
-// are extra column blocks in GEMM-1 and extra K blocks in GEMM-2).
+// A "group" is the shared experts (first; all T rows; their S sub-experts are extra column blocks
+// in GEMM-1 and extra K blocks in GEMM-2, which makes those the longest tiles) or a routed expert.
 //
 // CTA = 6 warps: warp 0 lane 0 issues TMA loads (A 128x64, B 256x64 or 128x64 bf16, 128-byte
 // swizzle) into a ring of 4 (6) stages; warp 1 lane 0 issues tcgen05.mma (M=128, N=256 or 128,
@@ -111,7 +111,8 @@ struct FfnSmemCtl {
   volatile int abort_flag;
   int n_groups;
   int total_tiles;
-  int tile_start[kMaxGroups + 1];   // first tile of each group
+  int shared_tiles;                 // tiles of the shared group: they come first in the tile numbering
+  int tile_start[kMaxGroups + 1];   // first tile of each routed group; [n_experts] = total_tiles
   int row_start[kMaxGroups];        // first row of each group in its A / output matrix
   int row_count[kMaxGroups];
   int mblock_start[kMaxGroups + 1]; // first row block of each group in the numbering of `done`
@@ -135,19 +136,40 @@ struct TileWalker {
     nb_routed = (p.n_per_sub + cols - 1) / cols;
     nb_shared = kSwiGLU ? nb_routed * p.shared_sub : nb_routed;
   }
+  // tile ids handed to one walker never decrease
   DEV TileCoord at(int tile, const FfnGemmParams& p) {
-    while (tile >= c->tile_start[g + 1]) ++g;   // tile < total_tiles, tile_start is non-decreasing
     TileCoord tc;
-    tc.group = g;
-    tc.shared = (g >= p.n_experts);
-    const int local = tile - c->tile_start[g];
-    const int mblocks = (c->row_count[g] + kTileM - 1) / kTileM;
+    tc.shared = tile < c->shared_tiles;
+    if (!tc.shared)
+      while (tile >= c->tile_start[g + 1]) ++g;   // tile < total_tiles, tile_start is non-decreasing
+    const int gi = tc.shared ? p.n_experts : g;
+    tc.group = gi;
+    const int local = tc.shared ? tile : tile - c->tile_start[gi];
+    const int mblocks = (c->row_count[gi] + kTileM - 1) / kTileM;
     tc.nb = local / mblocks;
     const int mb = local % mblocks;
-    tc.dep_id = c->mblock_start[g] + mb;
-    tc.m0 = c->row_start[g] + mb * kTileM;
-    tc.m_end = c->row_start[g] + c->row_count[g];
+    tc.dep_id = c->mblock_start[gi] + mb;
+    tc.m0 = c->row_start[gi] + mb * kTileM;
+    tc.m_end = c->row_start[gi] + c->row_count[gi];
     return tc;
+  }
+};
+
+// Which tiles a CTA (or CTA pair) works on, in order.  Normally tile c, c + G, c + 2G, ...  The shared
+// group's tiles come first in the numbering, and in GEMM-2 each of them runs S times as long as a
+// routed tile (K = S*I).  Handed out round-robin, the CTAs that got one would finish S - 1 tile
+// times after the others, alone on the memory system; so while the shared tiles fit one round
+// (n_sh <= G) the CTAs that hold one sit out the next w - 1 rounds of routed tiles (w = S).
+struct TileSched {
+  int c, G, n_sh, w;
+  bool skip;
+  DEV TileSched(int cta, int n_ctas, int shared_tiles, int weight)
+      : c(cta), G(n_ctas), n_sh(shared_tiles), w(weight), skip(shared_tiles <= n_ctas && weight > 1) {}
+  DEV int tile(int k) const {      // the CTA's k-th tile; increases with k; >= total_tiles ends the walk
+    if (!skip) return c + k * G;
+    const int free = G - n_sh;     // CTAs without a shared tile
+    if (c < n_sh) return k == 0 ? c : n_sh + w * free + c + (k - 1) * G;
+    return k < w ? c + k * free : n_sh + w * free + c + (k - w) * G;
   }
 };
 
@@ -199,15 +221,19 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   __syncthreads();
   if (tid == 0) {
     TileWalker<kSwiGLU, kN, kBM> w(ctl, p);
-    int acc = 0, mb_acc = 0;
-    for (int gi = 0; gi < n_groups; ++gi) {
+    // the shared group's tiles and row blocks are numbered first, the routed groups follow in order
+    const int sh_mblocks = p.shared_rows > 0 ? (p.shared_rows + kBM - 1) / kBM : 0;
+    int acc = sh_mblocks * w.nb_shared, mb_acc = sh_mblocks;
+    ctl->shared_tiles = acc;
+    ctl->mblock_start[p.n_experts] = 0;
+    for (int gi = 0; gi < p.n_experts; ++gi) {
       ctl->tile_start[gi] = acc;
       ctl->mblock_start[gi] = mb_acc;
       const int mblocks = (ctl->row_count[gi] + kBM - 1) / kBM;
-      acc += mblocks * (gi < p.n_experts ? w.nb_routed : w.nb_shared);
+      acc += mblocks * w.nb_routed;
       mb_acc += mblocks;
     }
-    ctl->tile_start[n_groups] = acc;
+    ctl->tile_start[p.n_experts] = acc;
     ctl->total_tiles = acc;
     ctl->n_groups = n_groups;
   }
@@ -216,6 +242,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   tc_fence_after_sync();
   const uint32_t tmem_base = ctl->tmem_base;
   const int total_tiles = ctl->total_tiles;
+  const TileSched sched((int)blockIdx.x, (int)gridDim.x, ctl->shared_tiles, kSwiGLU ? 1 : p.shared_sub);
   const int kb_routed = p.k_per_sub / kBK;
   const int kb_shared = kSwiGLU ? kb_routed : kb_routed * p.shared_sub;
   volatile int* abort_flag = &ctl->abort_flag;
@@ -229,7 +256,9 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
       TileWalker<kSwiGLU, kN, kBM> w(ctl, p);
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (int k = 0; ok; ++k) {
+        const int tile = sched.tile(k);
+        if (tile >= total_tiles) break;
         const TileCoord tc = w.at(tile, p);
         const CUtensorMap* tmA = tc.shared ? &tmA_shared : &tmA_routed;
         const CUtensorMap* tmB = tc.shared ? &tmB_shared : &tmB_routed;
@@ -294,7 +323,9 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
       constexpr uint32_t idesc = umma_idesc_bf16(kBM, kN);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+      for (int k = 0; ok; ++k, ++tcount) {
+        const int tile = sched.tile(k);
+        if (tile >= total_tiles) break;
         const TileCoord tc = w.at(tile, p);
         const int nkb = tc.shared ? kb_shared : kb_routed;
         const uint32_t a = tcount & 1u, aph = (tcount >> 1) & 1u;
@@ -325,7 +356,9 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
     const int q = warp & 3;                  // TMEM lane quarter this warp may read
     uint32_t tcount = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+    for (int k = 0; ok; ++k, ++tcount) {
+      const int tile = sched.tile(k);
+      if (tile >= total_tiles) break;
       const TileCoord tc = w.at(tile, p);
       const uint32_t a = tcount & 1u, aph = (tcount >> 1) & 1u;
       if (!(ok = mbar_wait_bounded_warp(&ctl->tmem_full[a], aph, abort_flag, p.dev_status))) break;
@@ -475,15 +508,19 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
   __syncthreads();
   if (tid == 0) {
     TileWalker<kSwiGLU, kN, kPairM> w(ctl, p);
-    int acc = 0, mb_acc = 0;
-    for (int gi = 0; gi < n_groups; ++gi) {
+    // the shared group's tiles and row blocks are numbered first, the routed groups follow in order
+    const int sh_mblocks = p.shared_rows > 0 ? (p.shared_rows + kPairM - 1) / kPairM : 0;
+    int acc = sh_mblocks * w.nb_shared, mb_acc = sh_mblocks;
+    ctl->shared_tiles = acc;
+    ctl->mblock_start[p.n_experts] = 0;
+    for (int gi = 0; gi < p.n_experts; ++gi) {
       ctl->tile_start[gi] = acc;
       ctl->mblock_start[gi] = mb_acc;
       const int mblocks = (ctl->row_count[gi] + kPairM - 1) / kPairM;
-      acc += mblocks * (gi < p.n_experts ? w.nb_routed : w.nb_shared);
+      acc += mblocks * w.nb_routed;
       mb_acc += mblocks;
     }
-    ctl->tile_start[n_groups] = acc;
+    ctl->tile_start[p.n_experts] = acc;
     ctl->total_tiles = acc;
     ctl->n_groups = n_groups;
   }
@@ -493,6 +530,7 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
   tc_fence_after_sync();
   const uint32_t tmem_base = ctl->tmem_base;
   const int total_tiles = ctl->total_tiles;
+  const TileSched sched(pair_id, n_pairs, ctl->shared_tiles, kSwiGLU ? 1 : p.shared_sub);
   const int kb_routed = p.k_per_sub / kBK;
   const int kb_shared = kSwiGLU ? kb_routed : kb_routed * p.shared_sub;
   volatile int* abort_flag = &ctl->abort_flag;
@@ -504,7 +542,9 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
       TileWalker<kSwiGLU, kN, kPairM> w(ctl, p);
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs) {
+      for (int k = 0; ok; ++k) {
+        const int tile = sched.tile(k);
+        if (tile >= total_tiles) break;
         const TileCoord tc = w.at(tile, p);
         const CUtensorMap* tmA = tc.shared ? &tmA_shared : &tmA_routed;
         const CUtensorMap* tmB = tc.shared ? &tmB_shared : &tmB_routed;
@@ -573,7 +613,9 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
       constexpr uint32_t idesc = umma_idesc_bf16(kPairM, kN);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs, ++tcount) {
+      for (int k = 0; ok; ++k, ++tcount) {
+        const int tile = sched.tile(k);
+        if (tile >= total_tiles) break;
         const TileCoord tc = w.at(tile, p);
         const int nkb = tc.shared ? kb_shared : kb_routed;
         const uint32_t a = tcount & 1u, aph = (tcount >> 1) & 1u;
@@ -604,7 +646,9 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
     const int q = warp & 3;
     uint32_t tcount = 0;
     bool ok = true;
-    for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs, ++tcount) {
+    for (int k = 0; ok; ++k, ++tcount) {
+      const int tile = sched.tile(k);
+      if (tile >= total_tiles) break;
       const TileCoord tc = w.at(tile, p);
       const uint32_t a = tcount & 1u, aph = (tcount >> 1) & 1u;
       if (!(ok = mbar_wait_bounded_warp(&ctl->tmem_full[a], aph, abort_flag, p.dev_status))) break;
