@@ -36,10 +36,10 @@ GATHER_ROWS_PER_EXPERT = 32     # the library's default: up to this many rows pe
 
 
 def kernels_per_layer(cfg, budget):
-    """Launches of one moe_layer_forward call: gate, routing (one fused launch up to 1024 tokens, else
+    """Launches of one moe_layer_forward call: gate, routing (one fused launch up to 8192 tokens, else
     select + permute count/scan/place), row gather (none where the expert GEMM fetches the rows of x
     itself), 2 expert GEMMs, combine."""
-    routing = 1 if cfg.T <= 1024 else 4
+    routing = 1 if cfg.T <= 8192 else 4
     gather = 0 if budget <= GATHER_ROWS_PER_EXPERT * cfg.N else 1
     return 1 + routing + gather + 2 + 1
 

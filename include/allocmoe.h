@@ -102,10 +102,11 @@ moe_status moe_permute(const moe_shape* shape, const uint16_t* x, const int32_t*
                        void* ws, size_t ws_bytes, void* stream);
 
 /* alloc_t_select and the list-building part of moe_permute (everything but the x_perm gather) in
- * one launch of one CTA: the form moe_layer_forward uses for T <= 1024, where four separate
- * launches cost more than the work.  Outputs are bit-identical to the two separate calls.
- * Supported when ceil(T/32) <= 32 and N * ceil(T/32) <= 40960; otherwise MOE_ERR_ARG.  Needs no
- * workspace. */
+ * one launch: one CTA up to 1024 tokens, a thread-block cluster of ceil(T/1024) CTAs that exchange
+ * their radix histograms and per-expert counts through distributed shared memory up to 8192 tokens.
+ * This is the form moe_layer_forward uses at those sizes, where four separate launches cost more
+ * than the work.  Outputs are bit-identical to the two separate calls.  T > 8192: MOE_ERR_ARG.
+ * Needs no workspace. */
 moe_status moe_route(const moe_shape* shape, const int32_t* topk_idx, const float* topk_score, int64_t budget,
                      int32_t* n_sel, int32_t* expert_offsets, int32_t* perm_token, float* perm_weight,
                      int32_t* pair_pos, int32_t* dev_status, void* stream);

@@ -20,6 +20,40 @@ struct SelectSmem {
   int bucket;
 };
 
+// One warp: given the histogram of the current 8-bit digit over the keys that share `prefix`, find the
+// digit in which the running count from the top first reaches *remaining, append it to the prefix,
+// and leave in *remaining the rank wanted inside that digit and in *bucket the digit's key count.
+DEV void radix_choose_digit(const int* hist, int shift, uint32_t prefix, uint32_t* prefix_out, int* remaining,
+                            int* bucket) {
+  const int lane = threadIdx.x & 31;
+  // lane l owns digits 255-8l .. 248-8l (descending)
+  int c[8], lsum = 0;
+#pragma unroll
+  for (int q = 0; q < 8; ++q) { c[q] = hist[255 - (lane * 8 + q)]; lsum += c[q]; }
+  int incl = lsum;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    int o = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += o;
+  }
+  int above = incl - lsum;           // keys in strictly higher digits than this lane's
+  const int rem = *remaining;
+  __syncwarp();
+  if (above < rem && rem <= incl) {  // exactly one lane
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      if (above < rem && rem <= above + c[q]) {
+        *prefix_out = prefix | ((uint32_t)(255 - (lane * 8 + q)) << shift);
+        *remaining = rem - above;
+        *bucket = c[q];              // keys that share the prefix chosen so far
+        above = rem;                 // stop
+      } else {
+        above += c[q];
+      }
+    }
+  }
+}
+
 // The selection, run by one CTA of kSelThreads threads.  `smem_raw`: sizeof(SelectSmem) bytes, then
 // room for the pool's keys when use_smem_keys is set.  Ends with a block-wide barrier after which
 // n_sel is visible to the whole CTA.
@@ -83,34 +117,7 @@ DEV void alloc_t_select_block(unsigned char* smem_raw, const float* __restrict__
       sm.hist[tid] = s;
     }
     __syncthreads();
-    if (warp == 0) {
-      // lane l owns digits 255-8l .. 248-8l (descending); find the digit where the running count
-      // from the top first reaches `remaining`.
-      int c[8], lsum = 0;
-#pragma unroll
-      for (int q = 0; q < 8; ++q) { c[q] = sm.hist[255 - (lane * 8 + q)]; lsum += c[q]; }
-      int incl = lsum;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        int o = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += o;
-      }
-      int above = incl - lsum;           // keys in strictly higher digits than this lane's
-      const int rem = sm.remaining;
-      if (above < rem && rem <= incl) {  // exactly one lane
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          if (above < rem && rem <= above + c[q]) {
-            sm.prefix = prefix | ((uint32_t)(255 - (lane * 8 + q)) << shift);
-            sm.remaining = rem - above;
-            sm.bucket = c[q];            // keys that share the prefix chosen so far
-            above = rem;                 // stop
-          } else {
-            above += c[q];
-          }
-        }
-      }
-    }
+    if (warp == 0) radix_choose_digit(sm.hist, shift, prefix, &sm.prefix, &sm.remaining, &sm.bucket);
     prefix_mask |= 255u << shift;
     __syncthreads();
   }
@@ -161,14 +168,16 @@ DEV void alloc_t_select_block(unsigned char* smem_raw, const float* __restrict__
 // ------------------------------------------------------------------ permutation
 constexpr int kMaxExperts = 128;
 
+// One warp, lane = token of the segment: mask[e] bit l set iff token l keeps expert e; e_out / n_out are
+// the lane's kept expert ids and their number.  n_raw < 0: the count is read from n_sel[t].
 DEV void build_masks(uint32_t* mask, const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ n_sel,
-                     int t, int T, int N, int K_orig, int lane, int (&e_out)[16], int& n_out) {
+                     int t, int T, int N, int K_orig, int lane, int (&e_out)[16], int& n_out, int n_known = -1) {
   for (int e = lane; e < N; e += 32) mask[e] = 0u;
   __syncwarp();
   n_out = 0;
   if (t < T) {
     // the count and all K_orig expert ids travel together (one round trip); ids past the count are ignored
-    const int n_raw = n_sel[t];
+    const int n_raw = n_known >= 0 ? n_known : n_sel[t];
 #pragma unroll
     for (int j = 0; j < 16; ++j) e_out[j] = (j < K_orig) ? topk_idx[(long long)t * K_orig + j] : 0;
     n_out = min(max(n_raw, 0), K_orig);
@@ -219,7 +228,7 @@ DEV void permute_scan_block(int32_t* seg_counts, int N, int nseg, long long budg
 DEV void permute_place_from_masks(const uint32_t* mask, const int (&e_loc)[16], int n,
                                   const float* __restrict__ topk_score, int seg, int T, int K_orig, int nseg,
                                   const int32_t* seg_base, long long budget, int32_t* __restrict__ perm_token,
-                                  float* __restrict__ perm_weight, int32_t* __restrict__ pair_pos);
+                                  float* __restrict__ perm_weight, int32_t* __restrict__ pair_pos, int base_col = -1);
 
 // One warp, one 32-token segment: list positions of its kept pairs.
 DEV void permute_place_warp(uint32_t* mask, const int32_t* __restrict__ topk_idx, const float* __restrict__ topk_score,
@@ -233,14 +242,16 @@ DEV void permute_place_warp(uint32_t* mask, const int32_t* __restrict__ topk_idx
                            pair_pos);
 }
 
-// The placement proper, from the segment's masks and this lane's expert ids (build_masks).
+// The placement proper, from the segment's masks and this lane's expert ids (build_masks).  The first list
+// position of (expert e, this segment) is seg_base[e * nseg + col], col = seg unless base_col is given.
 DEV void permute_place_from_masks(const uint32_t* mask, const int (&e_loc)[16], int n,
                                   const float* __restrict__ topk_score, int seg, int T, int K_orig, int nseg,
                                   const int32_t* seg_base, long long budget, int32_t* __restrict__ perm_token,
-                                  float* __restrict__ perm_weight, int32_t* __restrict__ pair_pos) {
+                                  float* __restrict__ perm_weight, int32_t* __restrict__ pair_pos, int base_col) {
   const int lane = threadIdx.x & 31;
   const int t = seg * 32 + lane;
   if (t >= T) return;
+  const int col = base_col >= 0 ? base_col : seg;
   const uint32_t lower = (1u << lane) - 1u;
   float w[16];   // all of the token's scores in one round trip
 #pragma unroll
@@ -251,7 +262,7 @@ DEV void permute_place_from_masks(const uint32_t* mask, const int (&e_loc)[16], 
     pos[j] = -1;
     if (j < n) {
       const int e = e_loc[j];
-      const int q = seg_base[(long long)e * nseg + seg] + __popc(mask[e] & lower);
+      const int q = seg_base[(long long)e * nseg + col] + __popc(mask[e] & lower);
       if (q >= 0 && q < budget) pos[j] = q;   // always true when sum n_sel == budget
     }
   }

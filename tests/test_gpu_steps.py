@@ -111,7 +111,13 @@ def test_moe_permute_bit_exact(T, N, K, kb, mult):
 @pytest.mark.parametrize("T,N,K,kb,mult,ties", [(1, 8, 2, 1, 1.0, False), (64, 8, 2, 0, 1.0, False),
                                                  (64, 64, 6, 1, 3.0, False), (333, 16, 4, 0, 1.3, True),
                                                  (1000, 64, 6, 1, 2.5, True), (1024, 128, 8, 2, 5.0, False),
-                                                 (1024, 64, 6, 1, 6.0, False), (1024, 64, 6, 1, 1.0, False)])
+                                                 (1024, 64, 6, 1, 6.0, False), (1024, 64, 6, 1, 1.0, False),
+                                                 # beyond 1024 tokens: a cluster of ceil(T/1024) CTAs
+                                                 (1025, 8, 2, 0, 1.5, True), (2048, 64, 6, 1, 3.0, False),
+                                                 (2500, 60, 4, 1, 2.5, True), (4096, 64, 6, 1, 3.0, True),
+                                                 (4096, 64, 6, 0, 2.0, False), (4100, 128, 8, 2, 5.0, True),
+                                                 (7000, 16, 16, 3, 9.7, True), (8192, 8, 2, 1, 1.5, False),
+                                                 (8192, 64, 8, 1, 8.0, False), (3000, 64, 6, 1, 1.0, False)])
 def test_moe_route_fused_bit_exact(T, N, K, kb, mult, ties):
     """The one-launch routing step gives what the oracle's selection and permutation give, ties included."""
     g = torch.Generator().manual_seed(T * 17 + N)
@@ -142,10 +148,10 @@ def test_moe_route_fused_bit_exact(T, N, K, kb, mult, ties):
 
 
 def test_moe_route_refuses_large_batches():
-    shape = B.make_shape(2048, 64, 64, 64, 0, 6, 1)
-    z = torch.zeros(2048 * 6, dtype=torch.int32, device="cuda")
+    shape = B.make_shape(8193, 64, 64, 64, 0, 6, 1)
+    z = torch.zeros(8193 * 6, dtype=torch.int32, device="cuda")
     with pytest.raises(B.MoeError) as ei:
-        B.moe_route(shape, z, z.float(), 4096, z, z, z, z.float(), z, _status())
+        B.moe_route(shape, z, z.float(), 16386, z, z, z, z.float(), z, _status())
     assert ei.value.status == B.MOE_ERR_ARG
 
 
