@@ -37,6 +37,78 @@ DEV void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// Softmax (fp32, expf) and sorted Top-K_orig for the tokens ks_rank*rows_per .. of the tile, from the KS partial
+// logit tiles rred[0..KS) (added in rank order, then the bias).  GS lanes work on one token, lane g of them owns
+// experts g, g+GS, ...; a warp finishes 32/GS tokens at a time.
+template <int NP, int NW, int GS>
+DEV void gate_finish(const float* const (&rred)[8], int KS, int ks_rank, int t0, int T, int N, int K_orig,
+                     const float* __restrict__ gate_bias, float* __restrict__ scores, int32_t* __restrict__ topk_idx,
+                     float* __restrict__ topk_score) {
+  constexpr int EPL = (NP + GS - 1) / GS, TPW = 32 / GS, RS = NP + 1, kGateTM = 16 * NW;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int rows_per = kGateTM / KS;
+  const int g8 = lane % GS, slot = lane / GS;
+  for (int rr0 = warp * TPW; rr0 < rows_per; rr0 += NW * TPW) {   // uniform across the warp
+    const int rr = rr0 + slot;
+    const int r = ks_rank * rows_per + rr;
+    const int t = t0 + r;
+    const bool valid = rr < rows_per && t < T;
+    float v[EPL];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int q = 0; q < EPL; ++q) {
+      const int e = g8 + GS * q;
+      float a = -INFINITY;
+      if (valid && e < N) {
+        a = rred[0][r * RS + e];
+#pragma unroll
+        for (int k = 1; k < 8; ++k)
+          if (k < KS) a += rred[k][r * RS + e];
+        if (gate_bias != nullptr) a += gate_bias[e];
+      }
+      v[q] = a;
+      mx = fmaxf(mx, v[q]);
+    }
+#pragma unroll
+    for (int d = GS / 2; d >= 1; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+    float sum = 0.f;
+#pragma unroll
+    for (int q = 0; q < EPL; ++q) {
+      v[q] = (valid && g8 + GS * q < N) ? expf(v[q] - mx) : 0.f;
+      sum += v[q];
+    }
+#pragma unroll
+    for (int d = GS / 2; d >= 1; d >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
+#pragma unroll
+    for (int q = 0; q < EPL; ++q) {
+      v[q] = valid ? v[q] / sum : 0.f;
+      const int e = g8 + GS * q;
+      if (scores != nullptr && valid && e < N) scores[(long long)t * N + e] = v[q];
+    }
+    uint32_t taken = 0u;
+    for (int j = 0; j < K_orig; ++j) {
+      float bv = -1.f;
+      int be = 0x7fffffff;
+#pragma unroll
+      for (int q = 0; q < EPL; ++q) {
+        const int e = g8 + GS * q;
+        if (e < N && !((taken >> q) & 1u) && v[q] > bv) { bv = v[q]; be = e; }   // ascending e: first max wins
+      }
+#pragma unroll
+      for (int d = GS / 2; d >= 1; d >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, d);
+        const int oe = __shfl_xor_sync(0xffffffffu, be, d);
+        if (ov > bv || (ov == bv && oe < be)) { bv = ov; be = oe; }
+      }
+      if (be % GS == g8 && be < N) taken |= 1u << (be / GS);
+      if (g8 == 0 && valid) {
+        topk_idx[(long long)t * K_orig + j] = be < N ? be : 0;
+        topk_score[(long long)t * K_orig + j] = bv;
+      }
+    }
+  }
+}
+
 // NT16 = number of 16-wide expert tiles (N padded to 16*NT16); NW = warps = 16-token slabs per CTA.
 template <int NT16, int NW>
 __global__ void __launch_bounds__(32 * NW)
@@ -139,72 +211,15 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
   }
   cluster.sync();   // every CTA's partial logits are in its red[0 .. 16*NW*RS)
 
-  // Softmax and sorted Top-K_orig.  This CTA finishes tokens ks_rank*32/KS .. of the tile, one warp
-  // per token at a time; lane l owns experts l, l+32, ...  The KS partial sums are added in rank
-  // order, then the bias.
-  constexpr int EPL = (NP + 31) / 32;
-  const int rows_per = kGateTM / KS;
+  // Softmax and sorted Top-K_orig of this CTA's share of the tile's tokens: eight lanes per token where a warp
+  // has at least four tokens to finish (large batches), else the whole warp on one token (fewer loads per lane).
   const float* rred[8];
 #pragma unroll
   for (int k = 0; k < 8; ++k) rred[k] = cluster.map_shared_rank(red, k < KS ? k : 0);
-  for (int rr = warp; rr < rows_per; rr += NW) {
-    const int r = ks_rank * rows_per + rr;
-    const int t = t0 + r;
-    if (t >= T) continue;   // uniform across the warp
-    float v[EPL];
-    float mx = -INFINITY;
-#pragma unroll
-    for (int q = 0; q < EPL; ++q) {
-      const int e = lane + 32 * q;
-      float a = -INFINITY;
-      if (e < N) {
-        a = rred[0][r * RS + e];
-#pragma unroll
-        for (int k = 1; k < 8; ++k)
-          if (k < KS) a += rred[k][r * RS + e];
-        if (gate_bias != nullptr) a += gate_bias[e];
-      }
-      v[q] = a;
-      mx = fmaxf(mx, v[q]);
-    }
-#pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
-    float sum = 0.f;
-#pragma unroll
-    for (int q = 0; q < EPL; ++q) {
-      v[q] = (lane + 32 * q < N) ? expf(v[q] - mx) : 0.f;
-      sum += v[q];
-    }
-#pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
-#pragma unroll
-    for (int q = 0; q < EPL; ++q) {
-      v[q] = v[q] / sum;
-      const int e = lane + 32 * q;
-      if (scores != nullptr && e < N) scores[(long long)t * N + e] = v[q];
-    }
-    uint32_t taken = 0u;
-    for (int j = 0; j < K_orig; ++j) {
-      float bv = -1.f;
-      int be = 0x7fffffff;
-#pragma unroll
-      for (int q = 0; q < EPL; ++q) {
-        const int e = lane + 32 * q;
-        if (e < N && !((taken >> q) & 1u) && v[q] > bv) { bv = v[q]; be = e; }   // ascending e: first max wins
-      }
-#pragma unroll
-      for (int d = 16; d >= 1; d >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, d);
-        const int oe = __shfl_xor_sync(0xffffffffu, be, d);
-        if (ov > bv || (ov == bv && oe < be)) { bv = ov; be = oe; }
-      }
-      if ((be & 31) == lane && be < N) taken |= 1u << (be >> 5);
-      if (lane == 0) {
-        topk_idx[(long long)t * K_orig + j] = be < N ? be : 0;
-        topk_score[(long long)t * K_orig + j] = bv;
-      }
-    }
-  }
+  if (kGateTM / KS >= NW * 4)
+    gate_finish<NP, NW, 8>(rred, KS, ks_rank, t0, T, N, K_orig, gate_bias, scores, topk_idx, topk_score);
+  else
+    gate_finish<NP, NW, 32>(rred, KS, ks_rank, t0, T, N, K_orig, gate_bias, scores, topk_idx, topk_score);
   cluster.sync();   // no CTA leaves while a peer may still read its partial sums
 }
 
