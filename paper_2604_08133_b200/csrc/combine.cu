@@ -15,7 +15,7 @@ DEV void fma8(float (&acc)[8], const uint4& v, float w) {
   }
 }
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 5)
 combine_kernel(const uint4* __restrict__ y_perm, const int32_t* __restrict__ pair_pos,
                const float* __restrict__ topk_score, const int32_t* __restrict__ n_sel,
                const uint4* __restrict__ y_shared, const uint4* __restrict__ x_res, int K_orig, int row_vec,
