@@ -282,13 +282,14 @@ def run_ours(args):
     x0 = layers[0]["x"]
     ws = B.new_workspace(shape, max(budgets))
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    bufs = [torch.empty_like(x0), torch.empty_like(x0)]
+    bufsets = [[torch.empty_like(x0), torch.empty_like(x0)] for _ in range(2)]   # second set: end-to-end pipeline
+    bufs = bufsets[0]
     xn = torch.empty_like(x0)
     stack = n_layers > 1     # the stack runs pre-norm: x_{l+1} = x_l + MoE_l(rmsnorm(x_l))
 
-    def layer(l, x, profile=None):
+    def layer(l, x, profile=None, p=0):
         d = layers[l]
-        out = bufs[l & 1]
+        out = bufsets[p][l & 1]
         xin = x
         if stack:
             B.moe_rmsnorm(shape, x, xn)
@@ -300,10 +301,10 @@ def run_ours(args):
                 profile[k] += v
         return out
 
-    def step(x_in=None):
+    def step(x_in=None, p=0):
         x = x0 if x_in is None else x_in
         for l in range(n_layers):
-            x = layer(l, x)
+            x = layer(l, x, p=p)
         return x
 
     def barrier():
@@ -411,22 +412,53 @@ def run_ours(args):
                                                   "whole DeepSeek-V2-Lite model, 1x H100 80GB, vLLM"}
             del ws_full
 
-        # ---- end to end: x from pinned host memory each step, out read back each step
+        # ---- end to end: every step's x comes from pinned host memory and its out goes back to pinned host
+        # memory.  Steps are independent batches, so the copies run on streams of their own and overlap the
+        # neighbouring steps' compute (two x buffers, two output sets); every step still pays both copies
+        # inside the timed region.
         x_host = x0.cpu().pin_memory()
-        out_host = torch.empty_like(x_host).pin_memory()
-        x_dev = torch.empty_like(x0)
+        out_host = [torch.empty_like(x_host).pin_memory() for _ in range(2)]
+        x_dev = [torch.empty_like(x0) for _ in range(2)]
+        cur = torch.cuda.current_stream()
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        ev_in = [torch.cuda.Event() for _ in range(2)]
+        ev_cmp = [torch.cuda.Event() for _ in range(2)]
+        ev_out = [torch.cuda.Event() for _ in range(2)]
 
-        def step_e2e():
-            x_dev.copy_(x_host, non_blocking=True)
-            y = step(x_dev)
-            out_host.copy_(y, non_blocking=True)
-        for _ in range(3):
-            step_e2e()
-        ms_e2e = timed(step_e2e, steps) / steps
+        def run_e2e(k):
+            s_in.wait_stream(cur)
+            s_out.wait_stream(cur)
+            for i in range(k):
+                p = i & 1
+                with torch.cuda.stream(s_in):
+                    if i >= 2:
+                        s_in.wait_event(ev_cmp[p])      # step i-2 has consumed x_dev[p]
+                    x_dev[p].copy_(x_host, non_blocking=True)
+                    ev_in[p].record(s_in)
+                cur.wait_event(ev_in[p])
+                if i >= 2:
+                    cur.wait_event(ev_out[p])           # step i-2's result has left output set p
+                y = step(x_dev[p], p)
+                ev_cmp[p].record(cur)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(ev_cmp[p])
+                    out_host[p].copy_(y, non_blocking=True)
+                    ev_out[p].record(s_out)
+            cur.wait_stream(s_in)
+            cur.wait_stream(s_out)
+        run_e2e(4)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        run_e2e(steps)
+        e1.record()
+        barrier()
+        ms_e2e = pdist.max_over_ranks(e0.elapsed_time(e1), device="cuda") / steps
         nbytes = x0.numel() * 2
         line["e2e"] = {"value": tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": nbytes,
                        "d2h_bytes_per_step": nbytes, "ms_per_step": ms_e2e,
-                       "note": "x copied from pinned host memory and out copied back every step; weights resident"}
+                       "note": "x copied from pinned host memory and out copied back every step on copy streams that "
+                               "overlap the neighbouring steps' compute; weights resident"}
         assert int(status.item()) == 0
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
