@@ -159,6 +159,8 @@ CONFIGS: Dict[str, MoEConfig] = {
     # stack of 26 such layers with per-layer budgets and a residual stream.
     "c4": MoEConfig("c4", T=2048, H=2048, N=64, I=1408, S=2, K_orig=6, K_base=1, budget=3 * 2048,
                     zipf_bias=True, n_layers=26),
+    # one layer of that stack on its own (profiling case for the mid-size regime: 96 rows per expert on average)
+    "c4l": MoEConfig("c4l", T=2048, H=2048, N=64, I=1408, S=2, K_orig=6, K_base=1, budget=3 * 2048, zipf_bias=True),
     # large-expert layer, prefill.
     "c5": MoEConfig("c5", T=8192, H=4096, N=8, I=14336, S=0, K_orig=2, K_base=1, budget=12288,
                     gate_scale=C5_GATE_SCALE),
