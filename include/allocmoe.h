@@ -143,7 +143,9 @@ moe_status moe_permute_static(const moe_shape* shape, const uint16_t* x, const i
  *   W13     device bf16 [N,2I,H]    rows 0..I-1 of an expert are W1, rows I..2I-1 are W3
  *   W2      device bf16 [N,H,I]
  *   y_perm  device bf16 [budget,H]
- * Experts with no rows read no weights. */
+ * Experts with no rows read no weights.  expert_offsets (device int32 [N+1]) is trusted to be
+ * non-decreasing within [0, budget]; values outside are clamped to that range on the device, so an
+ * inconsistent list gives meaningless rows but no access outside x_perm, y_perm or the workspace. */
 moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_perm,
                            const int32_t* expert_offsets, int64_t budget, const uint16_t* W13,
                            const uint16_t* W2, uint16_t* y_perm, int32_t* dev_status, void* ws,

@@ -52,6 +52,7 @@ constexpr int kMaxGroups = 130;     // up to 128 routed experts + the shared gro
 struct FfnGemmParams {
   const int32_t* expert_offsets;    // device [n_experts+1]; unused when n_experts == 0
   int n_experts;                    // routed groups
+  int routed_rows;                  // rows of the routed A / output matrices (the budget)
   int shared_rows;                  // T when the shared group is present, else 0
   int shared_sub;                   // S
   int n_per_sub;                    // output columns per (sub-)expert: I for GEMM-1, H for GEMM-2
@@ -65,6 +66,7 @@ struct FfnGemmParams {
   // of h it has finished (done[block], once per epilogue warp) and GEMM-2 loads a block's rows once
   // the count reaches dep_need_* (GEMM-1's tiles per block x epilogue warps).  nullptr = no tracking.
   int32_t* done;
+  int done_capacity;                // counters behind `done`; offsets that need more (inconsistent input) switch tracking off
   int dep_need_routed, dep_need_shared;
   // gather_rows > 0: the routed A tensor map has a box one row high and the producer warp fetches a
   // tile's rows four per TMA instruction, only those that hold rows of the expert's run.  GEMM-1 can
@@ -73,6 +75,7 @@ struct FfnGemmParams {
   // nullptr row m is row m (GEMM-2 on h).  gather_rows == 0: A rows come as one 128-row box.
   const int32_t* gather_idx;
   int gather_rows;
+  int gather_src_rows;              // rows of the matrix the indices point into; indices are clamped to it
 };
 
 // Token rows a producer lane fetches per stage when A is gathered: lane l owns rows 4l..4l+3 of the tile.
@@ -95,7 +98,8 @@ DEV GatherRows gather_rows_of_tile(const FfnGemmParams& p, int a_row, int m_end,
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int m = min(a_row + 4 * lane + i, p.gather_rows - 1);
-      g.r[i] = p.gather_idx != nullptr ? __ldg(p.gather_idx + m) : m;
+      // clamped: a routing step that reported an error may leave anything in the list
+      g.r[i] = p.gather_idx != nullptr ? min(max(__ldg(p.gather_idx + m), 0), p.gather_src_rows - 1) : m;
     }
   }
   return g;
@@ -111,6 +115,7 @@ struct FfnSmemCtl {
   volatile int abort_flag;
   int n_groups;
   int total_tiles;
+  int track_done;                   // the row-block counters are in use (FfnGemmParams::done, done_capacity)
   int shared_tiles;                 // tiles of the shared group: they come first in the tile numbering
   int tile_start[kMaxGroups + 1];   // first tile of each routed group; [n_experts] = total_tiles
   int row_start[kMaxGroups];        // first row of each group in its A / output matrix
@@ -210,9 +215,11 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   pdl_launch_dependents();   // expert_offsets and the operands come from earlier kernels of the stream
   for (int gi = tid; gi < n_groups; gi += kFfnThreads) {
     if (gi < p.n_experts) {
-      const int lo = p.expert_offsets[gi], hi = p.expert_offsets[gi + 1];
+      // clamped to the routed matrices' rows: a routing step that reported an error may leave anything here
+      const int lo = min(max(p.expert_offsets[gi], 0), p.routed_rows);
+      const int hi = min(max(p.expert_offsets[gi + 1], lo), p.routed_rows);
       ctl->row_start[gi] = lo;
-      ctl->row_count[gi] = max(hi - lo, 0);
+      ctl->row_count[gi] = hi - lo;
     } else {
       ctl->row_start[gi] = 0;
       ctl->row_count[gi] = p.shared_rows;
@@ -236,12 +243,15 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
     ctl->tile_start[p.n_experts] = acc;
     ctl->total_tiles = acc;
     ctl->n_groups = n_groups;
+    ctl->track_done = (p.done != nullptr && mb_acc <= p.done_capacity) ? 1 : 0;
   }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = ctl->tmem_base;
   const int total_tiles = ctl->total_tiles;
+  const bool track = ctl->track_done != 0;
+  if (!kSwiGLU && p.done != nullptr && !track) pdl_wait();   // no counters to go by: wait for all of GEMM-1
   const TileSched sched((int)blockIdx.x, (int)gridDim.x, ctl->shared_tiles, kSwiGLU ? 1 : p.shared_sub);
   const int kb_routed = p.k_per_sub / kBK;
   const int kb_shared = kSwiGLU ? kb_routed : kb_routed * p.shared_sub;
@@ -272,7 +282,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
         const bool gtile = gather && !tc.shared;
         GatherRows gr{};
         if (gtile) gr = gather_rows_of_tile(p, tc.m0, tc.m_end, lane, kBM);
-        if (!kSwiGLU && p.done != nullptr) {   // the block's rows of h are complete?
+        if (!kSwiGLU && track) {   // the block's rows of h are complete?
           if (lane == 0)
             ok = flag_wait_bounded(p.done + tc.dep_id, tc.shared ? p.dep_need_shared : p.dep_need_routed, abort_flag,
                                    p.dev_status);
@@ -417,7 +427,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
           }
         }
       }
-      if (kSwiGLU && p.done != nullptr) {   // publish this warp's quarter of the tile (FfnGemmParams::done)
+      if (kSwiGLU && track) {   // publish this warp's quarter of the tile (FfnGemmParams::done)
         __threadfence();
         __syncwarp();
         if (lane == 0) {
@@ -497,9 +507,11 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
   pdl_launch_dependents();
   for (int gi = tid; gi < n_groups; gi += kFfnThreads) {
     if (gi < p.n_experts) {
-      const int lo = p.expert_offsets[gi], hi = p.expert_offsets[gi + 1];
+      // clamped to the routed matrices' rows: a routing step that reported an error may leave anything here
+      const int lo = min(max(p.expert_offsets[gi], 0), p.routed_rows);
+      const int hi = min(max(p.expert_offsets[gi + 1], lo), p.routed_rows);
       ctl->row_start[gi] = lo;
-      ctl->row_count[gi] = max(hi - lo, 0);
+      ctl->row_count[gi] = hi - lo;
     } else {
       ctl->row_start[gi] = 0;
       ctl->row_count[gi] = p.shared_rows;
@@ -523,6 +535,7 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
     ctl->tile_start[p.n_experts] = acc;
     ctl->total_tiles = acc;
     ctl->n_groups = n_groups;
+    ctl->track_done = (p.done != nullptr && mb_acc <= p.done_capacity) ? 1 : 0;
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -530,6 +543,8 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
   tc_fence_after_sync();
   const uint32_t tmem_base = ctl->tmem_base;
   const int total_tiles = ctl->total_tiles;
+  const bool track = ctl->track_done != 0;
+  if (!kSwiGLU && p.done != nullptr && !track) pdl_wait();   // no counters to go by: wait for all of GEMM-1
   const TileSched sched(pair_id, n_pairs, ctl->shared_tiles, kSwiGLU ? 1 : p.shared_sub);
   const int kb_routed = p.k_per_sub / kBK;
   const int kb_shared = kSwiGLU ? kb_routed : kb_routed * p.shared_sub;
@@ -560,7 +575,7 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
         const bool gtile = gather && !tc.shared;
         GatherRows gr{};
         if (gtile) gr = gather_rows_of_tile(p, a_row, tc.m_end, lane, kBM);
-        if (!kSwiGLU && p.done != nullptr) {   // the block's rows of h are complete?
+        if (!kSwiGLU && track) {   // the block's rows of h are complete?
           if (lane == 0)
             ok = flag_wait_bounded(p.done + tc.dep_id, tc.shared ? p.dep_need_shared : p.dep_need_routed, abort_flag,
                                    p.dev_status);
@@ -706,7 +721,7 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
           }
         }
       }
-      if (kSwiGLU && p.done != nullptr) {   // publish this warp's quarter of the tile (FfnGemmParams::done)
+      if (kSwiGLU && track) {   // publish this warp's quarter of the tile (FfnGemmParams::done)
         __threadfence();
         __syncwarp();
         if (lane == 0) {
@@ -908,6 +923,7 @@ moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t*
   FfnGemmParams p{};
   p.expert_offsets = expert_offsets;
   p.n_experts = routed ? s->N : 0;
+  p.routed_rows = routed ? (int)budget : 0;
   p.shared_rows = shared ? s->T : 0;
   p.shared_sub = s->S;
   p.dev_status = dev_status;
@@ -918,12 +934,14 @@ moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t*
     const int per_tile = 4 * (pairs ? 2 : 1);                           // every epilogue warp counts once
     p.dep_need_routed = nb1 * per_tile;
     p.dep_need_shared = nb1 * s->S * per_tile;
+    p.done_capacity = (int)ffn_done_ints(s, routed ? budget : 0);
     if (cudaMemsetAsync(done, 0, ffn_done_ints(s, routed ? budget : 0) * sizeof(int32_t), stream) != cudaSuccess)
       return MOE_ERR_CUDA;
   }
   // GEMM-1
   p.gather_idx = routed ? gather_idx : nullptr;
   p.gather_rows = by_rows ? (int)budget : 0;
+  p.gather_src_rows = (int)s->T;
   p.n_per_sub = s->I;
   p.k_per_sub = s->H;
   p.up_row_offset = s->I;

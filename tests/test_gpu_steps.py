@@ -247,6 +247,34 @@ def test_grouped_ffn_skips_empty_experts_and_respects_segment_ends():
     assert max_rel(y[:T].float().cpu().numpy(), want) <= TOL_OUT
 
 
+def test_grouped_ffn_keeps_inconsistent_offsets_inside_the_list():
+    """Offsets that are negative, decreasing, past the list or overlapping (what a routing step that reported an error
+    may leave behind) are clamped to the list's rows: nothing is written outside y, and the next call is unaffected."""
+    T, H, N, I = 300, 128, 8, 128
+    cfg = synth.CONFIGS["c1"].with_(T=T, H=H, N=N, I=I)
+    d = synth.make_layer(cfg)
+    x_perm = d["x"].cuda()
+    shape = B.shape_of(cfg)
+    ws = B.new_workspace(shape, T)
+    st = _status()
+    W13, W2 = d["W13"].cuda(), d["W2"].cuda()
+    for bad in ([-5, 10, 5, 10 ** 6, 0, 0, 0, 0, 0], [0, T, 0, T, 0, T, 0, T, T], [0] + [T] * 8, [7 * T] * 9,
+                [0, 300, 300, 300, 300, 300, 300, 300, -1]):
+        y = torch.full((T + 8, H), 123.0, dtype=torch.bfloat16, device="cuda")
+        B.moe_grouped_ffn(shape, x_perm, torch.tensor(bad, dtype=torch.int32).cuda(), T, W13, W2, y, st, ws)
+        torch.cuda.synchronize()
+        assert st.item() == 0
+        assert (y[T:] == 123.0).all()
+    off = np.array([0, 100, 100, 100, 260, 260, 260, 260, 300], np.int32)
+    y = torch.full((T, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.moe_grouped_ffn(shape, x_perm, torch.from_numpy(off).cuda(), T, W13, W2, y, st, ws)
+    torch.cuda.synchronize()
+    xn, w13, w2 = np32(d["x"]), np32(d["W13"]), np32(d["W2"])
+    want = np.concatenate([orc.expert_ffn(xn[0:100], w13[0], w2[0]), orc.expert_ffn(xn[100:260], w13[3], w2[3]),
+                           orc.expert_ffn(xn[260:300], w13[7], w2[7])])
+    assert max_rel(y.float().cpu().numpy(), want) <= TOL_OUT
+
+
 @pytest.mark.parametrize("T,H,I,S", [(64, 256, 192, 2), (300, 128, 128, 1), (130, 256, 320, 3)])
 def test_shared_ffn_against_oracle(T, H, I, S):
     cfg = synth.CONFIGS["c2"].with_(T=T, H=H, N=8, I=I, S=S, K_orig=2, K_base=1, budget=T)
