@@ -412,6 +412,21 @@ def run_ours(args):
                                                   "whole DeepSeek-V2-Lite model, 1x H100 80GB, vLLM"}
             del ws_full
 
+        # ---- the same step replayed from a CUDA graph (one host call per step instead of one per kernel)
+        cur0 = torch.cuda.current_stream()
+        cap = torch.cuda.Stream()
+        cap.wait_stream(cur0)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(cap):
+            with torch.cuda.graph(graph, stream=cap):
+                step()
+        cur0.wait_stream(cap)
+        for _ in range(warmup):
+            graph.replay()
+        ms_graph = timed(graph.replay, steps) / steps
+        line["cuda_graph"] = {"ms_per_step": ms_graph, "value": tokens_per_step / (ms_graph * 1e-3), "unit": UNIT}
+        assert int(status.item()) == 0
+
         # ---- end to end: every step's x comes from pinned host memory and its out goes back to pinned host
         # memory.  Steps are independent batches, so the copies run on streams of their own and overlap the
         # neighbouring steps' compute (two x buffers, two output sets); every step still pays both copies

@@ -96,6 +96,44 @@ def test_forward_is_deterministic():
         assert torch.equal(ia["perm_token"], ib["perm_token"])
 
 
+@pytest.mark.parametrize("name", ["c2", "c4l"])
+def test_layer_forward_replays_from_a_cuda_graph(name):
+    """The call only enqueues work on the caller's stream (kernels as programmatic dependents, cluster launches, one
+    memset), so it can be captured once and replayed: same bits as the direct call, also after x changed in place."""
+    cfg = synth.CONFIGS[name]
+    if name == "c4l":
+        cfg = cfg.with_(T=1500, budget=3 * 1500)          # cluster routing kernel, ragged last segment
+    d = dev_layer(cfg)
+    shape = B.shape_of(cfg)
+    ws = B.new_workspace(shape, cfg.budget)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    x = d["x"].clone()
+    args = (shape, x, d["W_gate"], d["gate_bias"], d["W13"], d["W2"], d["Wsh13"], d["Wsh2"], cfg.budget)
+    want0 = torch.empty_like(x)
+    B.moe_layer_forward(*args, want0, status, ws)            # also the first call: one-time attribute set-up
+    out = torch.empty_like(x)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            B.moe_layer_forward(*args, out, status, ws)
+    torch.cuda.current_stream().wait_stream(side)
+    out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert torch.equal(out, want0)
+    x.copy_(torch.roll(d["x"], 7, dims=0))
+    want1 = torch.empty_like(x)
+    graph.replay()
+    B.moe_layer_forward(*args, want1, status, ws)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert torch.equal(out, want1)
+    assert not torch.equal(out, want0)
+
+
 def test_host_checked_errors_launch_nothing():
     cfg = synth.CONFIGS["c1"]
     d = dev_layer(cfg)
