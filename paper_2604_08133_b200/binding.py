@@ -148,7 +148,7 @@ def alloc_l_solve(S, B: int):
 
 def moe_route(shape, topk_idx, topk_score, budget, n_sel, expert_offsets, perm_token, perm_weight, pair_pos, dev_status,
               stream=None):
-    """alloc_t_select + the list-building part of moe_permute in one launch (T <= 1024)."""
+    """alloc_t_select + the list-building part of moe_permute in one launch (T <= 8192)."""
     _check("moe_route", lib().moe_route(ctypes.byref(shape), _p(topk_idx), _p(topk_score), int(budget), _p(n_sel),
                                         _p(expert_offsets), _p(perm_token), _p(perm_weight), _p(pair_pos),
                                         _p(dev_status), _stream(stream)))

@@ -1,5 +1,6 @@
 // Fused routing step of moe_layer_forward: Alloc-T selection (Sec. 3.3) and the permutation's
-// count / scan / place in ONE launch of one CTA.
+// count / scan / place in ONE launch -- of one CTA up to 1024 tokens (moe_route_kernel), of a
+// thread-block cluster of 1024-token CTAs up to 8192 tokens (moe_route_cluster_kernel, below).
 //
 // Each of the four steps is a few microseconds of work for a single CTA at the sizes a layer call
 // sees (at most a few tens of thousands of (token, expert) pairs); launched separately they cost
