@@ -18,6 +18,9 @@
 // K=16) into one of two TMEM accumulators; warps 2-5 read the finished accumulator with
 // tcgen05.ld, apply the epilogue and store bf16 rows (row-masked at the ragged end of an expert's
 // run) while the next tile's main loop runs.  Every wait is bounded (see common.cuh).
+// Where expert runs are short (FfnGemmParams::gather_rows) the A rows do not come as one 128-row box:
+// the 32 lanes of warp 0 fetch four rows each with tile::gather4 loads -- for GEMM-1 straight from x
+// through perm_token, so no permuted copy of x exists -- and skip the rows past the run's end.
 //
 // Two variants of the kernel: one CTA per 128-row tile (ffn_gemm_kernel) and a CTA pair per 256-row
 // tile (ffn_gemm_pair_kernel, tcgen05 cta_group::2); launch_ffn picks by shape.  GEMM-2 is launched
