@@ -181,6 +181,42 @@ struct TileSched {
   }
 };
 
+// One warp: first tile and first row block of every group from the groups' row counts (the shared group's tiles
+// and row blocks are numbered first, the routed groups follow in order; every routed group has nb_routed column
+// blocks).  Lane l takes a run of consecutive experts, a warp scan joins the runs.
+template <int kTileM>
+DEV void build_tile_table(FfnSmemCtl* ctl, const FfnGemmParams& p, int nb_routed, int nb_shared, int n_groups) {
+  const int lane = threadIdx.x & 31;
+  const int sh_mblocks = p.shared_rows > 0 ? (p.shared_rows + kTileM - 1) / kTileM : 0;
+  const int sh_tiles = sh_mblocks * nb_shared;
+  const int per = (p.n_experts + 31) / 32;
+  const int g0 = min(lane * per, p.n_experts), g1 = min(g0 + per, p.n_experts);
+  int mb = 0;
+  for (int g = g0; g < g1; ++g) mb += (ctl->row_count[g] + kTileM - 1) / kTileM;
+  int incl = mb;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int o = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += o;
+  }
+  int before = incl - mb;   // routed row blocks of lower experts
+  for (int g = g0; g < g1; ++g) {
+    ctl->mblock_start[g] = sh_mblocks + before;
+    ctl->tile_start[g] = sh_tiles + before * nb_routed;
+    before += (ctl->row_count[g] + kTileM - 1) / kTileM;
+  }
+  const int routed_mblocks = __shfl_sync(0xffffffffu, incl, 31);
+  if (lane == 0) {
+    const int total = sh_tiles + routed_mblocks * nb_routed;
+    ctl->shared_tiles = sh_tiles;
+    ctl->mblock_start[p.n_experts] = 0;
+    ctl->tile_start[p.n_experts] = total;
+    ctl->total_tiles = total;
+    ctl->n_groups = n_groups;
+    ctl->track_done = (p.done != nullptr && sh_mblocks + routed_mblocks <= p.done_capacity) ? 1 : 0;
+  }
+}
+
 template <bool kSwiGLU, int kN>
 __global__ void __launch_bounds__(kFfnThreads, 1)
 ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_routed,
@@ -229,24 +265,9 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
     }
   }
   __syncthreads();
-  if (tid == 0) {
+  if (warp == 2) {
     TileWalker<kSwiGLU, kN, kBM> w(ctl, p);
-    // the shared group's tiles and row blocks are numbered first, the routed groups follow in order
-    const int sh_mblocks = p.shared_rows > 0 ? (p.shared_rows + kBM - 1) / kBM : 0;
-    int acc = sh_mblocks * w.nb_shared, mb_acc = sh_mblocks;
-    ctl->shared_tiles = acc;
-    ctl->mblock_start[p.n_experts] = 0;
-    for (int gi = 0; gi < p.n_experts; ++gi) {
-      ctl->tile_start[gi] = acc;
-      ctl->mblock_start[gi] = mb_acc;
-      const int mblocks = (ctl->row_count[gi] + kBM - 1) / kBM;
-      acc += mblocks * w.nb_routed;
-      mb_acc += mblocks;
-    }
-    ctl->tile_start[p.n_experts] = acc;
-    ctl->total_tiles = acc;
-    ctl->n_groups = n_groups;
-    ctl->track_done = (p.done != nullptr && mb_acc <= p.done_capacity) ? 1 : 0;
+    build_tile_table<kBM>(ctl, p, w.nb_routed, w.nb_shared, n_groups);
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -521,24 +542,9 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
     }
   }
   __syncthreads();
-  if (tid == 0) {
+  if (warp == 2) {
     TileWalker<kSwiGLU, kN, kPairM> w(ctl, p);
-    // the shared group's tiles and row blocks are numbered first, the routed groups follow in order
-    const int sh_mblocks = p.shared_rows > 0 ? (p.shared_rows + kPairM - 1) / kPairM : 0;
-    int acc = sh_mblocks * w.nb_shared, mb_acc = sh_mblocks;
-    ctl->shared_tiles = acc;
-    ctl->mblock_start[p.n_experts] = 0;
-    for (int gi = 0; gi < p.n_experts; ++gi) {
-      ctl->tile_start[gi] = acc;
-      ctl->mblock_start[gi] = mb_acc;
-      const int mblocks = (ctl->row_count[gi] + kPairM - 1) / kPairM;
-      acc += mblocks * w.nb_routed;
-      mb_acc += mblocks;
-    }
-    ctl->tile_start[p.n_experts] = acc;
-    ctl->total_tiles = acc;
-    ctl->n_groups = n_groups;
-    ctl->track_done = (p.done != nullptr && mb_acc <= p.done_capacity) ? 1 : 0;
+    build_tile_table<kPairM>(ctl, p, w.nb_routed, w.nb_shared, n_groups);
   }
   tc_fence_before_sync();
   __syncthreads();
