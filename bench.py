@@ -27,8 +27,8 @@ UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel (expert GEMM-1), from the ncu
 # captures summarised under profiles/ (workload, budget) -> bytes; absent = not captured for the current kernel.
 NCU_TRAFFIC_BYTES = {
-    ("c2", 192): 716.0e6 + 4.4e6,        # profiles/ffn_gemm_c2_decode.md
-    ("c3", 12288): 832.3e6 + 55.8e6,     # profiles/ffn_gemm_c3_prefill.md
+    ("c2", 192): 716.0e6 + 4.6e6,        # profiles/ffn_gemm_c2_decode.md
+    ("c3", 12288): 830.6e6 + 55.4e6,     # profiles/ffn_gemm_c3_prefill.md
 }
 
 
