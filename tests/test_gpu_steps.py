@@ -318,18 +318,19 @@ def test_combine_against_oracle_formula():
     assert max_rel(got, want) <= 4e-3
 
 
-@pytest.mark.parametrize("pair,gather", [("0", "0"), ("1", "0"), ("0", "1000000"), ("1", "1000000")])
-def test_expert_gemm_variants_forced(pair, gather):
+@pytest.mark.parametrize("pair,gather,tile_n", [("0", "0", "256"), ("1", "0", "256"), ("0", "1000000", "256"),
+                                                 ("1", "1000000", "256"), ("0", "0", "128"), ("0", "1000000", "128")])
+def test_expert_gemm_variants_forced(pair, gather, tile_n):
     """The library picks one-CTA or CTA-pair tiles, and box loads or row-by-row fetches of the token rows (from a
-    permuted copy or straight from x through perm_token), by shape; every combination must be right on every shape.
-    The choices are read from the environment once per process, so each forced setting runs the expert-GEMM tests and
-    the small whole-layer tests in a process of its own."""
+    permuted copy or straight from x through perm_token), by shape; every combination must be right on every shape,
+    and so must the 128-row weight tile kept behind its knob.  The choices are read from the environment once per
+    process, so each forced setting runs the expert-GEMM tests and the small whole-layer tests in a process of its own."""
     import os
     import subprocess
     import sys
     if os.environ.get("ALLOCMOE_PAIR") is not None:
         pytest.skip("already inside a forced run")
-    env = dict(os.environ, ALLOCMOE_PAIR=pair, ALLOCMOE_GATHER=gather)
+    env = dict(os.environ, ALLOCMOE_PAIR=pair, ALLOCMOE_GATHER=gather, ALLOCMOE_TILE_N=tile_n)
     here = os.path.dirname(os.path.abspath(__file__))
     r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(here, "test_gpu_steps.py"),
                         os.path.join(here, "test_gpu_layer.py"), "-m", "gpu", "-q", "-x", "-k",
