@@ -276,6 +276,10 @@ def test_other_model_shapes(name, T, mult):
     (257, 256, 8, 64, 3, 4, 4, 1028),       # K_base = K_orig: nothing to redistribute, three shared experts
     (300, 128, 8, 128, 2, 4, 1, 1200),      # budget = K_orig*T: plain Top-K_orig
     (700, 128, 4 * 2, 256, 1, 2, 1, 1390),  # ~174 rows per expert: the CTA-pair tiles, with a shared expert
+    (1030, 64, 16, 64, 0, 4, 1, 2000),      # just past 1024 tokens: routing cluster whose second CTA holds 6 tokens
+    (2100, 128, 128, 64, 1, 16, 3, 9000),   # routing cluster of 3 CTAs at the largest N and K_orig; row-indexed A loads
+    (1500, 64, 8, 128, 3, 2, 0, 1600),      # three shared sub-experts (GEMM-2 tiles of triple length), K_base 0
+    (40, 320, 20, 448, 2, 5, 1, 41),        # budget one above K_base*T: a single redistributed pair
 ])
 def test_odd_shapes(T, H, N, I, S, K, kb, budget):
     cfg = synth.MoEConfig("odd", T=T, H=H, N=N, I=I, S=S, K_orig=K, K_base=kb, budget=budget, zipf_bias=(N >= 12), seed=T)
