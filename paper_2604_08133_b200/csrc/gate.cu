@@ -212,12 +212,15 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
   cluster.sync();   // every CTA's partial logits are in its red[0 .. 16*NW*RS)
 
   // Softmax and sorted Top-K_orig of this CTA's share of the tile's tokens: eight lanes per token where a warp
-  // has at least four tokens to finish (large batches), else the whole warp on one token (fewer loads per lane).
+  // has at least four tokens to finish (large batches), sixteen where it has two, else the whole warp on one
+  // token (fewer loads per lane).
   const float* rred[8];
 #pragma unroll
   for (int k = 0; k < 8; ++k) rred[k] = cluster.map_shared_rank(red, k < KS ? k : 0);
   if (kGateTM / KS >= NW * 4)
     gate_finish<NP, NW, 8>(rred, KS, ks_rank, t0, T, N, K_orig, gate_bias, scores, topk_idx, topk_score);
+  else if (kGateTM / KS >= NW * 2)
+    gate_finish<NP, NW, 16>(rred, KS, ks_rank, t0, T, N, K_orig, gate_bias, scores, topk_idx, topk_score);
   else
     gate_finish<NP, NW, 32>(rred, KS, ks_rank, t0, T, N, K_orig, gate_bias, scores, topk_idx, topk_score);
   cluster.sync();   // no CTA leaves while a peer may still read its partial sums
