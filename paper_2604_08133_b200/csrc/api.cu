@@ -6,7 +6,7 @@
 
 // launchers defined next to their kernels
 moe_status launch_moe_gate(const moe_shape*, const uint16_t*, const uint16_t*, const float*, float*, int32_t*, float*,
-                           cudaStream_t);
+                           int32_t*, int, cudaStream_t);
 moe_status launch_alloc_t_select(const moe_shape*, const float*, int64_t, int32_t*, int32_t*, cudaStream_t);
 moe_status launch_moe_permute(const moe_shape*, const uint16_t*, const int32_t*, const float*, const int32_t*, int64_t,
                               int32_t*, int32_t*, float*, int32_t*, uint16_t*, int32_t*, int32_t*, cudaStream_t);
@@ -16,7 +16,7 @@ moe_status launch_moe_route(const moe_shape*, const float*, const int32_t*, int6
                             int32_t*, int32_t*, cudaStream_t);
 moe_status launch_ffn(const moe_shape*, const uint16_t*, const int32_t*, const int32_t*, int64_t, const uint16_t*, const uint16_t*,
                       uint16_t*, uint16_t*, const uint16_t*, const uint16_t*, const uint16_t*, uint16_t*, uint16_t*,
-                      int32_t*, int32_t*, cudaStream_t, cudaEvent_t);
+                      int32_t*, int32_t*, bool, cudaStream_t, cudaEvent_t);
 size_t ffn_done_ints(const moe_shape*, int64_t);
 bool ffn_gathers(const moe_shape*, int64_t);
 moe_status launch_moe_combine(const moe_shape*, const uint16_t*, const int32_t*, const float*, const int32_t*,
@@ -112,7 +112,7 @@ moe_status moe_gate(const moe_shape* shape, const uint16_t* x, const uint16_t* W
                     float* scores, int32_t* topk_idx, float* topk_score, void* stream) {
   if (!shape_ok(shape) || !x || !W_gate || !topk_idx || !topk_score) return MOE_ERR_ARG;
   if (!aligned16(x) || !aligned16(W_gate) || !aligned16(topk_idx) || !aligned16(topk_score)) return MOE_ERR_ARG;
-  return launch_moe_gate(shape, x, W_gate, gate_bias, scores, topk_idx, topk_score, (cudaStream_t)stream);
+  return launch_moe_gate(shape, x, W_gate, gate_bias, scores, topk_idx, topk_score, nullptr, 0, (cudaStream_t)stream);
 }
 
 moe_status alloc_t_select(const moe_shape* shape, const float* topk_score, int64_t budget, int32_t* n_sel,
@@ -163,7 +163,7 @@ moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_perm, const
   const WsLayout L = ws_layout(shape, budget);
   if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
   return launch_ffn(shape, x_perm, nullptr, expert_offsets, budget, W13, W2, at<uint16_t>(ws, L.h), y_perm, nullptr, nullptr,
-                    nullptr, nullptr, nullptr, dev_status, at<int32_t>(ws, L.gemm_done), (cudaStream_t)stream, nullptr);
+                    nullptr, nullptr, nullptr, dev_status, at<int32_t>(ws, L.gemm_done), false, (cudaStream_t)stream, nullptr);
 }
 
 moe_status moe_shared_ffn(const moe_shape* shape, const uint16_t* x, const uint16_t* Wsh13, const uint16_t* Wsh2,
@@ -173,8 +173,8 @@ moe_status moe_shared_ffn(const moe_shape* shape, const uint16_t* x, const uint1
   const WsLayout L = ws_layout(shape, 0);
   if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
   return launch_ffn(shape, nullptr, nullptr, nullptr, 0, nullptr, nullptr, nullptr, nullptr, x, Wsh13, Wsh2,
-                    at<uint16_t>(ws, L.h_sh), y_shared, dev_status, at<int32_t>(ws, L.gemm_done), (cudaStream_t)stream,
-                    nullptr);
+                    at<uint16_t>(ws, L.h_sh), y_shared, dev_status, at<int32_t>(ws, L.gemm_done), false,
+                    (cudaStream_t)stream, nullptr);
 }
 
 moe_status moe_combine(const moe_shape* shape, const uint16_t* y_perm, const int32_t* pair_pos,
@@ -215,7 +215,9 @@ moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const ui
   if (ffn_gathers(shape, budget)) x_perm = nullptr;
 
   prof_mark(0, st);
-  moe_status r = launch_moe_gate(shape, x, W_gate, gate_bias, nullptr, topk_idx, topk_score, st);
+  // the gate launch also clears the expert GEMMs' row-block counters (no memset between kernels of the call)
+  moe_status r = launch_moe_gate(shape, x, W_gate, gate_bias, nullptr, topk_idx, topk_score, at<int32_t>(ws, L.gemm_done),
+                                 (int)ffn_done_ints(shape, budget), st);
   if (r != MOE_OK) return r;
   prof_mark(1, st);
   if (moe_route_fits(shape)) {
@@ -237,7 +239,7 @@ moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const ui
   r = launch_ffn(shape, x_perm != nullptr ? x_perm : x, x_perm != nullptr ? nullptr : perm_token, expert_offsets, budget,
                  W13, W2, at<uint16_t>(ws, L.h), y_perm,
                  shape->S > 0 ? x : nullptr, Wsh13, Wsh2, at<uint16_t>(ws, L.h_sh), y_shared, dev_status,
-                 at<int32_t>(ws, L.gemm_done), st, g_prof_on ? g_prof_ev[4] : nullptr);
+                 at<int32_t>(ws, L.gemm_done), true, st, g_prof_on ? g_prof_ev[4] : nullptr);
   if (r != MOE_OK) return r;
   prof_mark(5, st);
   r = launch_moe_combine(shape, y_perm, pair_pos, topk_score, n_sel, y_shared, residual, budget, out,

@@ -895,11 +895,12 @@ bool ffn_gathers(const moe_shape* s, int64_t budget) {
 //   routed part present iff budget > 0 && x_perm != nullptr; shared part iff S > 0 && x_shared != nullptr.
 //   gather_idx != nullptr: x_perm is x [T, H] itself and routed row m is x[gather_idx[m]] (perm_token);
 //   callers pass it only where ffn_gathers() holds.
+//   done_is_clear: an earlier kernel of the stream has zeroed `done` (else a memset is enqueued here).
 moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t* gather_idx,
                       const int32_t* expert_offsets, int64_t budget,
                       const uint16_t* W13, const uint16_t* W2, uint16_t* h, uint16_t* y_perm, const uint16_t* x_shared,
                       const uint16_t* Wsh13, const uint16_t* Wsh2, uint16_t* h_sh, uint16_t* y_shared,
-                      int32_t* dev_status, int32_t* done, cudaStream_t stream, cudaEvent_t between) {
+                      int32_t* dev_status, int32_t* done, bool done_is_clear, cudaStream_t stream, cudaEvent_t between) {
   const bool routed = (budget > 0 && x_perm != nullptr);
   const bool shared = (s->S > 0 && x_shared != nullptr);
   if (!routed && !shared) return MOE_OK;
@@ -944,7 +945,8 @@ moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t*
     p.dep_need_routed = nb1 * per_tile;
     p.dep_need_shared = nb1 * s->S * per_tile;
     p.done_capacity = (int)ffn_done_ints(s, routed ? budget : 0);
-    if (cudaMemsetAsync(done, 0, ffn_done_ints(s, routed ? budget : 0) * sizeof(int32_t), stream) != cudaSuccess)
+    if (!done_is_clear &&
+        cudaMemsetAsync(done, 0, ffn_done_ints(s, routed ? budget : 0) * sizeof(int32_t), stream) != cudaSuccess)
       return MOE_ERR_CUDA;
   }
   // GEMM-1

@@ -114,7 +114,8 @@ template <int NT16, int NW>
 __global__ void __launch_bounds__(32 * NW)
 moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ W_gate,
                 const float* __restrict__ gate_bias, int T, int H, int N, int K_orig, int w_stride,
-                float* __restrict__ scores, int32_t* __restrict__ topk_idx, float* __restrict__ topk_score) {
+                float* __restrict__ scores, int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
+                int32_t* __restrict__ zero_ptr, int zero_n) {
   cg::cluster_group cluster = cg::this_cluster();
   const int KS = (int)cluster.num_blocks();        // CTAs per token tile (cluster spans blockIdx.y)
   const int ks_rank = (int)cluster.block_rank();
@@ -130,6 +131,11 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
   const int nchunks = (nchunks_all - ks_rank + KS - 1) / KS;   // this CTA's chunks: ks_rank, ks_rank + KS, ...
   const int n_vec = N / 8;   // 16-byte pieces per W_gate row
   pdl_prologue_done();
+  // Side job for the layer call: clear the expert GEMMs' row-block counters.  As the first kernel of the call this
+  // one runs after everything that read them; doing it here keeps a memset out of the stream, which would sit
+  // between two kernels and stop the later one from starting early as a programmatic dependent.
+  if (zero_ptr != nullptr && blockIdx.x == 0 && blockIdx.y == 0)
+    for (int i = tid; i < zero_n; i += kGateThreads) zero_ptr[i] = 0;
 
   auto issue = [&](int chunk) {
     if (chunk < nchunks) {
@@ -238,7 +244,8 @@ static int gate_w_stride(int NP) {
 
 template <int NT16, int NW>
 static moe_status gate_launch_t(const moe_shape* s, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,
-                                float* scores, int32_t* topk_idx, float* topk_score, cudaStream_t stream) {
+                                float* scores, int32_t* topk_idx, float* topk_score, int32_t* zero_ptr, int zero_n,
+                                cudaStream_t stream) {
   constexpr int NP = NT16 * 16, TM = 16 * NW;
   const int w_stride = gate_w_stride(NP);
   size_t pipe = (size_t)kGateStages * (TM * kGateXStride * 2 + kGateKC * w_stride * 2);
@@ -260,29 +267,33 @@ static moe_status gate_launch_t(const moe_shape* s, const uint16_t* x, const uin
   const cudaError_t err = launch_dependent(
       moe_gate_kernel<NT16, NW>, dim3((unsigned)tiles, (unsigned)ks, 1), dim3(32 * NW), smem, stream, (unsigned)ks,
       reinterpret_cast<const __nv_bfloat16*>(x), reinterpret_cast<const __nv_bfloat16*>(W_gate), gate_bias, (int)s->T,
-      (int)s->H, (int)s->N, (int)s->K_orig, w_stride, scores, topk_idx, topk_score);
+      (int)s->H, (int)s->N, (int)s->K_orig, w_stride, scores, topk_idx, topk_score, zero_ptr, zero_n);
   return err == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 template <int NT16>
 static moe_status gate_launch_nw(const moe_shape* s, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,
-                                 float* scores, int32_t* topk_idx, float* topk_score, cudaStream_t stream) {
-  if (s->T >= 2048) return gate_launch_t<NT16, 4>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-  return gate_launch_t<NT16, 2>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+                                 float* scores, int32_t* topk_idx, float* topk_score, int32_t* zero_ptr, int zero_n,
+                                 cudaStream_t stream) {
+  if (s->T >= 2048)
+    return gate_launch_t<NT16, 4>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
+  return gate_launch_t<NT16, 2>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
 }
 
+// zero_ptr / zero_n: device ints the launch also clears (nullptr: none)
 moe_status launch_moe_gate(const moe_shape* s, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,
-                           float* scores, int32_t* topk_idx, float* topk_score, cudaStream_t stream) {
+                           float* scores, int32_t* topk_idx, float* topk_score, int32_t* zero_ptr, int zero_n,
+                           cudaStream_t stream) {
   const int nt16 = (s->N + 15) / 16;
   switch (nt16) {
-    case 1: return gate_launch_nw<1>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-    case 2: return gate_launch_nw<2>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-    case 3: return gate_launch_nw<3>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-    case 4: return gate_launch_nw<4>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-    case 5: return gate_launch_nw<5>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-    case 6: return gate_launch_nw<6>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-    case 7: return gate_launch_nw<7>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
-    case 8: return gate_launch_nw<8>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, stream);
+    case 1: return gate_launch_nw<1>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
+    case 2: return gate_launch_nw<2>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
+    case 3: return gate_launch_nw<3>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
+    case 4: return gate_launch_nw<4>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
+    case 5: return gate_launch_nw<5>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
+    case 6: return gate_launch_nw<6>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
+    case 7: return gate_launch_nw<7>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
+    case 8: return gate_launch_nw<8>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
     default: return MOE_ERR_ARG;
   }
 }
