@@ -6,13 +6,21 @@
 
 A step is one moe_layer_forward call (gate GEMM + softmax + Top-K, Alloc-T selection,
 permutation, grouped SwiGLU expert GEMMs + shared experts, combine) over one batch of seeded
-synthetic tokens.  The default workload is the DeepSeek-V2-Lite-shaped decode layer (c2).
+synthetic tokens.  The headline workload is the DeepSeek-V2-Lite-shaped decode layer (c2); on one
+GPU the same line also carries the prefill layer (c3 at 3xT), the large-expert layer (c5) and the
+26-layer stack (c4) under "workloads", each timed the same way.
+
+Timing: W warm-up steps, then blocks of exactly K steps, each block bracketed by a barrier and a
+device synchronisation and timed with CUDA events (max over ranks); blocks are repeated until at
+least 5 have run and they add up to half a second, and the median block gives ms_per_step.
 One JSON line is printed by rank 0.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
+import math
 import os
 import sys
 import threading
@@ -24,12 +32,36 @@ if ROOT not in sys.path:
 
 METRIC = "budgeted MoE-layer tokens/s"
 UNIT = "tokens/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel (expert GEMM-1), from the ncu
-# captures summarised under profiles/ (workload, budget) -> bytes; absent = not captured for the current kernel.
-NCU_TRAFFIC_BYTES = {
-    ("c2", 192): 716.0e6 + 4.6e6,        # profiles/ffn_gemm_c2_decode.md
-    ("c3", 12288): 830.6e6 + 55.4e6,     # profiles/ffn_gemm_c3_prefill.md
-}
+MIN_BLOCKS = 5            # timed blocks per figure, at least
+MIN_REGION_S = 0.5        # and at least this much timed work in total
+MAX_BLOCKS = 400
+
+
+def kernel_source_sha16():
+    """Fingerprint of the expert-GEMM kernels' source: ncu counters are only quoted for the code they were taken on."""
+    h = hashlib.sha256()
+    for f in ("ffn.cu", "common.cuh"):
+        with open(os.path.join(ROOT, "paper_2604_08133_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic_bytes(kernel, workload, budget):
+    """dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of `kernel` on this workload, from the table of
+    ncu captures kept with the profile summaries (tab-separated: kernel, workload, budget, bytes per launch, source
+    fingerprint, commit, how it was taken).  None when there is no capture of the kernel source as it stands."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    sha = kernel_source_sha16()
+    with open(path) as f:
+        for ln in f:
+            if ln.startswith("#") or not ln.strip():
+                continue
+            c = ln.rstrip("\n").split("\t")
+            if len(c) >= 5 and kernel.startswith(c[0]) and c[1] == workload and int(c[2]) == int(budget) and c[4] == sha:
+                return float(c[3])
+    return None
 
 
 GATHER_ROWS_PER_EXPERT = 32     # the library's default: up to this many rows per routed expert GEMM-1 reads x by index
@@ -58,6 +90,10 @@ def parse_args():
                          "on a seeded synthetic sensitivity matrix (same total)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the stage profile / full-Top-K / e2e passes")
+    ap.add_argument("--no-workloads", action="store_true", help="headline workload only (no c3 / c5 / c4 entries)")
+    ap.add_argument("--global-alloc-t", action="store_true",
+                    help="also time the batch-wide Alloc-T path (gate, all-gather of the score rows, selection over "
+                         "the whole pool, routed layer call); always on with more than one GPU")
     return ap.parse_args()
 
 
@@ -170,7 +206,7 @@ def time_oracle(cfg, budget, steps=1, warmup=0, target_tokens=None):
         orc.layer_forward(*a)
     t0 = time.perf_counter()
     for _ in range(steps):
-        orc.layer_forward(*a)
+        last = orc.layer_forward(*a)
     dt = (time.perf_counter() - t0) / steps
     cores = torch.get_num_threads()
     try:
@@ -180,7 +216,8 @@ def time_oracle(cfg, budget, steps=1, warmup=0, target_tokens=None):
         pass
     sample = (f"oracle layer_forward on the first {Ts} of {cfg.T} tokens, budget {b}"
               if Ts < cfg.T else f"oracle layer_forward on the whole batch (T={cfg.T}, budget {b})")
-    return dict(value=Ts / dt, unit=UNIT, cores=int(cores), kind="oracle", sample=sample, s_per_step=dt, tokens=Ts)
+    return dict(value=Ts / dt, unit=UNIT, cores=int(cores), kind="oracle", sample=sample, s_per_step=dt, tokens=Ts,
+                budget=b, result=last)
 
 
 def oracle_tokens_for(cfg):
@@ -245,28 +282,84 @@ def gemm1_work(cfg, budget, touched):
     return flops, by
 
 
-def run_ours(args):
+SECONDARY = (("c3", None), ("c5", None), ("c4", None))     # (workload, budget multiple; None = the workload's own)
+
+
+class Env:
+    """Process-group facts and the timing primitives shared by every measurement of a run."""
+
+    def __init__(self):
+        import torch
+        import torch.distributed as dist
+        self.torch, self.dist = torch, dist
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        torch.cuda.set_device(self.local)
+        if self.world > 1:
+            dist.init_process_group("nccl", device_id=torch.device("cuda", self.local))
+
+    def barrier(self):
+        if self.world > 1:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def time_block(self, fn, k):
+        """k calls of fn between a barrier + synchronize on both sides, CUDA events, max over ranks; ms."""
+        from paper_2604_08133_b200 import dist as pdist
+        torch = self.torch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        self.barrier()
+        e0.record()
+        for _ in range(k):
+            fn()
+        e1.record()
+        self.barrier()
+        return pdist.max_over_ranks(e0.elapsed_time(e1), device="cuda")
+
+    def time_blocks(self, fn, k, call_is_k_steps=False):
+        """Blocks of exactly k steps until MIN_BLOCKS have run and they add up to MIN_REGION_S.  Returns the
+        per-step ms of every block.  call_is_k_steps: fn() itself runs the k steps (a pipelined loop)."""
+        one = (lambda: self.time_block(fn, 1)) if call_is_k_steps else (lambda: self.time_block(fn, k))
+        first = one()
+        n = max(MIN_BLOCKS, int(math.ceil(MIN_REGION_S * 1e3 / max(first, 1e-3))))
+        n = min(n, MAX_BLOCKS)
+        ms = [first] + [one() for _ in range(n - 1)]
+        return [m / k for m in ms]
+
+
+def median(v):
+    s = sorted(v)
+    return s[len(s) // 2] if len(s) % 2 else 0.5 * (s[len(s) // 2 - 1] + s[len(s) // 2])
+
+
+def default_steps(cfg):
+    """Steps per block when --steps is not given: blocks of roughly 0.1 s."""
+    if cfg.n_layers > 1:
+        return 10, 3
+    if cfg.T <= 256:
+        return 500, 50
+    return (25, 5) if cfg.H * cfg.I > 2e7 else (200, 20)
+
+
+def bench_workload(env, args, name, budget_mult, steps_arg, warmup_arg, full=True):
+    """All figures of one workload on this rank's GPU; `full` adds the CUDA-graph and end-to-end passes."""
     import torch
-    import torch.distributed as dist
     from paper_2604_08133_b200 import binding as B
-    from paper_2604_08133_b200 import dist as pdist
     from paper_2604_08133_b200 import synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    B.lib()   # fails loudly when the CUDA library is missing
-
-    cfg, budget = workload_cfg(args)
+    class A:      # the argument view workload_cfg() expects
+        pass
+    a = A()
+    a.workload, a.budget_mult = name, budget_mult
+    a.k_base = args.k_base if name == args.workload else None
+    cfg, budget = workload_cfg(a)
     # every rank works on its own batch (independent problems, replicated weights): weak scaling
-    cfg = cfg.with_(seed=cfg.seed + rank)
+    cfg = cfg.with_(seed=cfg.seed + env.rank)
     n_layers = cfg.n_layers
-    steps = args.steps if args.steps is not None else (2000 if cfg.T <= 256 else (20 if n_layers > 1 else 300))
-    warmup = args.warmup if args.warmup is not None else (50 if cfg.T <= 256 else (3 if n_layers > 1 else 20))
-    warmup = max(3, warmup)
+    dsteps, dwarm = default_steps(cfg)
+    steps = steps_arg if steps_arg is not None else dsteps
+    warmup = max(3, warmup_arg if warmup_arg is not None else dwarm)
 
     shape = B.shape_of(cfg)
     layers = [synth.make_layer(cfg, l, device="cuda", with_x=(l == 0)) for l in range(n_layers)]
@@ -283,7 +376,6 @@ def run_ours(args):
     ws = B.new_workspace(shape, max(budgets))
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     bufsets = [[torch.empty_like(x0), torch.empty_like(x0)] for _ in range(2)]   # second set: end-to-end pipeline
-    bufs = bufsets[0]
     xn = torch.empty_like(x0)
     stack = n_layers > 1     # the stack runs pre-norm: x_{l+1} = x_l + MoE_l(rmsnorm(x_l))
 
@@ -307,44 +399,28 @@ def run_ours(args):
             x = layer(l, x, p=p)
         return x
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def timed(fn, k):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        e0.record()
-        for _ in range(k):
-            fn()
-        e1.record()
-        barrier()
-        return pdist.max_over_ranks(e0.elapsed_time(e1), device="cuda")
-
     for _ in range(warmup):
         step()
-    sampler = ClockSampler(local)
-    barrier()
+    sampler = ClockSampler(env.local)
+    env.barrier()
     sampler.start()
-    ms = timed(step, steps)
+    per_step = env.time_blocks(step, steps)
     clocks = sampler.stop()
     assert int(status.item()) == 0, "device status %d" % int(status.item())
-    ms_per_step = ms / steps
-    tokens_per_step = cfg.T * world
-    value = tokens_per_step / (ms_per_step * 1e-3)
-
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
+    ms_per_step = median(per_step)
+    tokens_per_step = cfg.T * env.world
+    per_step_launches = sum(kernels_per_layer(cfg, b) + (1 if stack else 0) for b in budgets)
+    res = {
+        "value": tokens_per_step / (ms_per_step * 1e-3), "unit": UNIT, "ms_per_step": ms_per_step,
+        "steps": steps, "warmup": warmup, "blocks": len(per_step),
+        "timed_region_s": sum(per_step) * steps * 1e-3, "ms_per_step_min": min(per_step), "ms_per_step_max": max(per_step),
         "config": {"workload": describe(cfg, budgets[0] if n_layers == 1 else sum(budgets) // n_layers),
                    "layers": n_layers, "parallelism": "independent batches per GPU, replicated weights, no collective",
                    "l2": "weights exceed L2 (no flush)" if (cfg.N + cfg.S) * 6 * cfg.H * cfg.I > 126e6 else
                          "L2-resident workload, no flush (latency-bound case)"},
-        "clocks": clocks, "gpu_launches": sum(kernels_per_layer(cfg, b) + (1 if stack else 0) for b in budgets) * steps,
+        "clocks": clocks, "gpu_launches": per_step_launches * steps * len(per_step),
+        "launches_per_step": per_step_launches,
     }
-
     peaks = load_peaks()
     if not args.no_extras:
         # ---- touched experts (data dependent) from the last call's offsets
@@ -352,10 +428,11 @@ def run_ours(args):
         off = inter["expert_offsets"].cpu()
         touched = int((off[1:] > off[:-1]).sum())
 
-        # ---- stage profile: the same steps again with events at the stage boundaries
+        # ---- stage profile: the same steps again with events at the stage boundaries (the dominant kernel's
+        # average launch duration, measured live on the stream it is launched on)
         B.moe_profile_enable(True)
         acc = {k: 0.0 for k in B.PROFILE_STAGES}
-        nprof = min(steps, 200)
+        nprof = max(3, min(steps * len(per_step), int(0.25e3 / max(ms_per_step, 1e-3)), 400))
         for _ in range(3):
             step()
         for _ in range(nprof):
@@ -377,41 +454,44 @@ def run_ours(args):
         else:
             roof = {"bound": "tensor", "achieved": g_flops / t_g1 / 1e12, "peak": peaks["bf16_tflops_sustained"],
                     "unit": "TFLOP/s"}
+            roof["frac_of_burst_peak"] = roof["achieved"] / peaks["bf16_tflops"]
         roof["frac"] = roof["achieved"] / roof["peak"]
-        roof["traffic"] = NCU_TRAFFIC_BYTES.get((cfg.name, int(budgets[0]))) if n_layers == 1 else None
         pair = 128 * cfg.N < b_mean <= 256 * cfg.N      # the library's own rule for CTA-pair tiles
-        roof["kernel"] = ("ffn_gemm_pair_kernel<true>" if pair else "ffn_gemm_kernel<true, 256>") + \
-            " (expert GEMM-1 + SwiGLU, routed and shared groups)"
+        kname = "ffn_gemm_pair_kernel<true>" if pair else "ffn_gemm_kernel<true, 256>"
+        roof["traffic"] = ncu_traffic_bytes(kname, cfg.name, int(budgets[0])) if n_layers == 1 else None
+        roof["kernel"] = kname + " (expert GEMM-1 + SwiGLU, routed and shared groups)"
         roof["peak_source"] = peaks["source"] + (" (sustained bf16)" if roof["bound"] == "tensor" else " (copy)")
         roof["avg_launch_ms"] = stage_ms["ffn_gemm1"]
+        roof["launches_timed"] = nprof * n_layers
         roof["algorithmic_bytes"] = g_bytes
         roof["algorithmic_flops"] = g_flops
-        line["roofline"] = roof
-        line["stage_ms"] = stage_ms
-        line["touched_experts"] = touched
-        line["layer_roofline"] = {"flops": flops, "bytes": by, "t_flop_us": t_flop * 1e6, "t_byte_us": t_byte * 1e6,
-                                  "bound": "tensor" if t_flop > t_byte else "hbm",
-                                  "frac": max(t_flop, t_byte) / (ms_per_step * 1e-3 / n_layers),
-                                  "tokens_per_s_at_roofline": cfg.T / max(t_flop, t_byte) / n_layers}
+        res["roofline"] = roof
+        res["stage_ms"] = stage_ms
+        res["touched_experts"] = touched
+        res["layer_roofline"] = {"flops": flops, "bytes": by, "t_flop_us": t_flop * 1e6, "t_byte_us": t_byte * 1e6,
+                                 "bound": "tensor" if t_flop > t_byte else "hbm",
+                                 "frac": max(t_flop, t_byte) / (ms_per_step * 1e-3 / n_layers),
+                                 "tokens_per_s_at_roofline": cfg.T / max(t_flop, t_byte) / n_layers}
 
         # ---- the same kernels at the full Top-K_orig budget (budgeted-vs-full speedup)
         if n_layers == 1 and budget < cfg.K_orig * cfg.T:
-            full = cfg.K_orig * cfg.T
-            ws_full = B.new_workspace(shape, full)
-            out_f = bufs[0]
+            full_b = cfg.K_orig * cfg.T
+            ws_full = B.new_workspace(shape, full_b)
+            out_f = bufsets[0][0]
             d = layers[0]
 
             def step_full():
                 B.moe_layer_forward(shape, x0, d["W_gate"], d["gate_bias"], d["W13"], d["W2"], d["Wsh13"], d["Wsh2"],
-                                    full, out_f, status, ws_full)
+                                    full_b, out_f, status, ws_full)
             for _ in range(warmup):
                 step_full()
-            ms_full = timed(step_full, steps) / steps
-            line["full_topk"] = {"budget": full, "ms_per_step": ms_full, "speedup_budgeted_vs_full": ms_full / ms_per_step,
-                                 "paper_context": "paper reports 1.15x prefill / 1.34x decode at half budget, "
-                                                  "whole DeepSeek-V2-Lite model, 1x H100 80GB, vLLM"}
+            ms_full = median(env.time_blocks(step_full, steps))
+            res["full_topk"] = {"budget": full_b, "ms_per_step": ms_full, "speedup_budgeted_vs_full": ms_full / ms_per_step,
+                                "paper_context": "paper reports 1.15x prefill / 1.34x decode at half budget, "
+                                                 "whole DeepSeek-V2-Lite model, 1x H100 80GB, vLLM"}
             del ws_full
 
+    if full and not args.no_extras:
         # ---- the same step replayed from a CUDA graph (one host call per step instead of one per kernel)
         cur0 = torch.cuda.current_stream()
         cap = torch.cuda.Stream()
@@ -423,8 +503,8 @@ def run_ours(args):
         cur0.wait_stream(cap)
         for _ in range(warmup):
             graph.replay()
-        ms_graph = timed(graph.replay, steps) / steps
-        line["cuda_graph"] = {"ms_per_step": ms_graph, "value": tokens_per_step / (ms_graph * 1e-3), "unit": UNIT}
+        ms_graph = median(env.time_blocks(graph.replay, steps))
+        res["cuda_graph"] = {"ms_per_step": ms_graph, "value": tokens_per_step / (ms_graph * 1e-3), "unit": UNIT}
         assert int(status.item()) == 0
 
         # ---- end to end: every step's x comes from pinned host memory and its out goes back to pinned host
@@ -462,29 +542,123 @@ def run_ours(args):
             cur.wait_stream(s_in)
             cur.wait_stream(s_out)
         run_e2e(4)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        e0.record()
-        run_e2e(steps)
-        e1.record()
-        barrier()
-        ms_e2e = pdist.max_over_ranks(e0.elapsed_time(e1), device="cuda") / steps
+        ms_e2e = median(env.time_blocks(lambda: run_e2e(steps), steps, call_is_k_steps=True))
         nbytes = x0.numel() * 2
-        line["e2e"] = {"value": tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": nbytes,
-                       "d2h_bytes_per_step": nbytes, "ms_per_step": ms_e2e,
-                       "note": "x copied from pinned host memory and out copied back every step on copy streams that "
-                               "overlap the neighbouring steps' compute; weights resident"}
+        res["e2e"] = {"value": tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": nbytes,
+                      "d2h_bytes_per_step": nbytes, "ms_per_step": ms_e2e,
+                      "note": "x copied from pinned host memory and out copied back every step on copy streams that "
+                              "overlap the neighbouring steps' compute; weights resident"}
         assert int(status.item()) == 0
 
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        r = time_oracle(cfg, budgets[0], steps=1, warmup=0, target_tokens=oracle_tokens_for(cfg))
+    if (args.global_alloc_t or env.world > 1) and n_layers == 1 and name == args.workload:
+        res["global_alloc_t"] = bench_global_alloc_t(env, cfg, shape, layers[0], budget, steps, warmup)
+    res["_cfg"], res["_budget"] = cfg, budgets[0]
+    return res
+
+
+def bench_global_alloc_t(env, cfg, shape, d, budget, steps, warmup):
+    """The batch-wide Alloc-T (Sec. 3.3 pools the scores of ALL tokens) with the batch sharded over the ranks:
+    gate -> all-gather of the score rows -> selection over the whole pool on every rank -> routed layer call.
+    Reports the whole layer and, separately, what the exchange adds: (gate + all-gather + selection) - gate."""
+    import torch
+    from paper_2604_08133_b200 import binding as B
+    from paper_2604_08133_b200 import dist as pdist
+    lay = pdist.GlobalAllocTLayer(shape, "cuda", always_collective=True)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = torch.empty_like(d["x"])
+    budget_global = budget * env.world
+
+    def layer_step():
+        lay.forward(d["x"], d["W_gate"], d["gate_bias"], d["W13"], d["W2"], d["Wsh13"], d["Wsh2"], budget_global, out, st)
+
+    def route_step():
+        lay.route(d["x"], d["W_gate"], d["gate_bias"], budget_global, st)
+
+    def gate_step():
+        B.moe_gate(shape, d["x"], d["W_gate"], d["gate_bias"], None, lay.topk_idx, lay.topk_score)
+
+    r = {}
+    for key, fn in (("layer_ms", layer_step), ("gate_exchange_select_ms", route_step), ("gate_ms", gate_step)):
+        for _ in range(warmup):
+            fn()
+        r[key] = median(env.time_blocks(fn, steps))
+    assert int(st.item()) == 0, "device status %d" % int(st.item())
+    r["exchange_select_ms"] = r["gate_exchange_select_ms"] - r["gate_ms"]
+    r["value"] = cfg.T * env.world / (r["layer_ms"] * 1e-3)
+    r["unit"] = UNIT
+    r["pool_keys"] = cfg.T * env.world * (cfg.K_orig - cfg.K_base)
+    r["exchange"] = ("all_gather_into_tensor of %d fp32 score rows per rank over NCCL" % cfg.T) if \
+        (env.world > 1 or env.dist.is_initialized()) else "one rank, no process group: the collective is skipped"
+    return r
+
+
+def parity_on_sample(cfg, budget, ref):
+    """The GPU path against the oracle on the sample the CPU baseline timed (ref: the oracle's layer_forward
+    result on the first Ts tokens): tokens whose selection differs (near-ties between the GPU's fp32 and the
+    oracle's fp64 scores) and the output error measures on all other tokens."""
+    import numpy as np
+    import torch
+    from paper_2604_08133_b200 import binding as B
+    from paper_2604_08133_b200 import synth
+    Ts = ref["out"].shape[0]
+    scfg = cfg.with_(T=Ts)
+    d = synth.make_layer(cfg, device="cuda")
+    x = d["x"][:Ts].contiguous()
+    shape = B.shape_of(scfg)
+    ws = B.new_workspace(shape, budget)
+    out = torch.empty_like(x)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.moe_layer_forward(shape, x, d["W_gate"], d["gate_bias"], d["W13"], d["W2"], d["Wsh13"], d["Wsh2"], budget, out, st, ws)
+    torch.cuda.synchronize()
+    inter = B.moe_layer_intermediates(shape, budget, ws)
+    same = (ref["n_sel"] == inter["n_sel"].cpu().numpy()) & (ref["topk_idx"] == inter["topk_idx"].cpu().numpy()).all(axis=1)
+    got = out.float().cpu().numpy().astype(np.float64)[same]
+    want = np.asarray(ref["out"], np.float64)[same]
+    dlt = np.abs(got - want)
+    rms = max(float(np.sqrt((want * want).mean())), 1e-30)
+    return {"tokens": int(Ts), "flips": int((~same).sum()), "dev_status": int(st.item()),
+            "max_rel": float(dlt.max() / max(np.abs(want).max(), 1e-30)),
+            "elementwise": float((dlt / (np.abs(want) + rms)).max()),
+            "rms_rel": float(np.sqrt((dlt * dlt).mean()) / rms),
+            "note": "GPU vs the fp64 oracle on the CPU baseline's sample; flips = tokens whose kept set differs "
+                    "(score near-ties), outputs compared on the others"}
+
+
+def run_ours(args):
+    import torch
+    from paper_2604_08133_b200 import binding as B
+    env = Env()
+    B.lib()   # fails loudly when the CUDA library is missing
+
+    res = bench_workload(env, args, args.workload, args.budget_mult, args.steps, args.warmup, full=True)
+    cfg, budget0 = res.pop("_cfg"), res.pop("_budget")
+    line = {"metric": METRIC, "value": res.pop("value"), "unit": res.pop("unit"), "n_gpus": env.world,
+            "steps": res.pop("steps"), "warmup": res.pop("warmup"), "ms_per_step": res.pop("ms_per_step"),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic"}
+    line.update(res)
+
+    if env.world == 1 and not args.no_workloads and not args.no_extras and args.workload == "c2" \
+            and args.budget_mult is None and args.k_base is None:
+        line["workloads"] = {}
+        for name, mult in SECONDARY:
+            torch.cuda.empty_cache()
+            r = bench_workload(env, args, name, mult, None, None, full=False)
+            r.pop("_cfg"), r.pop("_budget")
+            line["workloads"][name] = r
+
+    if env.rank == 0 and env.world == 1 and not args.no_cpu_baseline:
+        torch.cuda.empty_cache()
+        r = time_oracle(cfg, budget0, steps=1, warmup=0, target_tokens=oracle_tokens_for(cfg))
         line["cpu_baseline"] = {"value": r["value"], "unit": UNIT, "cores": r["cores"], "kind": "oracle",
                                 "sample": r["sample"]}
-    if rank == 0:
+        line["parity"] = parity_on_sample(cfg, r["budget"], r["result"])
+    if env.rank == 0:
         print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
+    if env.world > 1:
+        env.dist.barrier()
+        env.dist.destroy_process_group()
+
+
 
 
 def main():

@@ -89,7 +89,10 @@ moe_status alloc_t_select(const moe_shape* shape, const float* topk_score, int64
                           int32_t* n_sel, int32_t* dev_status, void* ws, size_t ws_bytes,
                           void* stream);
 
-/* Lists the kept pairs expert-ascending and token-ascending inside an expert.
+/* Permutation of the kept (token, expert) pairs into per-expert segments: the step between Alloc-T's
+ * selection (Sec. 3.3) and the per-expert feed-forward executions of Sec. 3.1.  The paper names no such
+ * step -- it masks the scores and leaves the dispatch to the serving stack; the order below is this
+ * library's choice.  Lists the kept pairs expert-ascending and token-ascending inside an expert.
  *   expert_offsets device int32 [N+1]   exclusive prefix of per-expert counts, [N] = budget
  *   perm_token     device int32 [budget] token of each listed pair
  *   perm_weight    device fp32  [budget] its routing score
@@ -135,18 +138,23 @@ moe_status moe_permute_static(const moe_shape* shape, const uint16_t* x, const i
                               int32_t* pair_pos, uint16_t* x_perm, int32_t* dev_status,
                               void* stream);
 
-/* Routed experts ("each activated expert corresponds to one feed-forward execution",
- * Sec. 3.1).  For every listed pair p of expert e:
+/* Routed experts: one expert feed-forward execution per kept (token, expert) pair (Sec. 3.1, the cost
+ * model behind the activation budget).  For every listed pair p of expert e:
  *   h = silu(x_p W1_e^T) * (x_p W3_e^T)  (fp32 accumulation, h stored as bf16)
  *   y_perm[p] = h W2_e^T                 (fp32 accumulation, stored as bf16)
- *   x_perm  device bf16 [budget,H]  rows in list order (moe_permute's x_perm)
+ *   x_or_xperm device bf16: with perm_token == NULL the rows in list order, [budget,H] (moe_permute's
+ *              x_perm); with perm_token given the tokens themselves, x [T,H], and row p is
+ *              x[perm_token[p]] -- read by index straight from x where expert runs are short (at most 32
+ *              rows per expert on average), gathered once into the workspace otherwise
+ *   perm_token device int32 [budget] or NULL
  *   W13     device bf16 [N,2I,H]    rows 0..I-1 of an expert are W1, rows I..2I-1 are W3
  *   W2      device bf16 [N,H,I]
  *   y_perm  device bf16 [budget,H]
  * Experts with no rows read no weights.  expert_offsets (device int32 [N+1]) is trusted to be
- * non-decreasing within [0, budget]; values outside are clamped to that range on the device, so an
- * inconsistent list gives meaningless rows but no access outside x_perm, y_perm or the workspace. */
-moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_perm,
+ * non-decreasing within [0, budget]; values outside are clamped to that range on the device, and so are
+ * the entries of perm_token to [0, T), so an inconsistent list gives meaningless rows but no access
+ * outside x, y_perm or the workspace. */
+moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_or_xperm, const int32_t* perm_token,
                            const int32_t* expert_offsets, int64_t budget, const uint16_t* W13,
                            const uint16_t* W2, uint16_t* y_perm, int32_t* dev_status, void* ws,
                            size_t ws_bytes, void* stream);
@@ -165,8 +173,9 @@ moe_status moe_combine(const moe_shape* shape, const uint16_t* y_perm, const int
                        const float* topk_score, const int32_t* n_sel, const uint16_t* y_shared,
                        uint16_t* out, void* stream);
 
-/* The whole layer on one stream: moe_gate, alloc_t_select, moe_permute, moe_grouped_ffn
- * (+ moe_shared_ffn when S > 0), moe_combine; all intermediates live in `ws`.
+/* The whole budgeted layer (Eq. 1, Alloc-T of Sec. 3.3 / Eq. 8-10, Eq. 2) on one stream: moe_gate,
+ * alloc_t_select, moe_permute, moe_grouped_ffn (+ moe_shared_ffn when S > 0), moe_combine; all
+ * intermediates live in `ws`.
  * Wsh13 / Wsh2 are ignored when S == 0.
  *   residual  device bf16 [T,H] or NULL: added to the result, out = residual + MoE(x) (fp32 add,
  *             one bf16 rounding): the step of a residual layer stack.  May alias x, not out. */
@@ -175,6 +184,23 @@ moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const ui
                              const uint16_t* Wsh13, const uint16_t* Wsh2, int64_t budget,
                              const uint16_t* residual, uint16_t* out, int32_t* dev_status, void* ws,
                              size_t ws_bytes, void* stream);
+
+/* The layer from a selection the caller already holds: permutation, experts and Eq. 2 for the given
+ * Top-K_orig rows and kept counts.  This is the local part of Alloc-T over a batch that is sharded across
+ * GPUs (Sec. 3.3 pools the scores of all tokens): each rank runs moe_gate, the ranks exchange their score
+ * rows, every rank runs alloc_t_select on the whole pool and hands its own slice of n_sel to this call.
+ * How many pairs this rank keeps is then known to the device only, so the call takes an upper bound:
+ *   n_sel       device int32 [T], values in [0, K_orig]
+ *   budget_max  upper bound of sum n_sel; sizes the workspace (moe_workspace_bytes(shape, budget_max)).
+ *               A larger sum raises MOE_ERR_BUDGET in dev_status; every access stays in bounds.
+ *   budget_hint expected sum (0: budget_max); only picks between kernel variants, any value is correct
+ * Everything else as for moe_layer_forward.  Nothing is read back to the host. */
+moe_status moe_layer_forward_routed(const moe_shape* shape, const uint16_t* x, const int32_t* topk_idx,
+                                    const float* topk_score, const int32_t* n_sel, int64_t budget_max,
+                                    int64_t budget_hint, const uint16_t* W13, const uint16_t* W2,
+                                    const uint16_t* Wsh13, const uint16_t* Wsh2, const uint16_t* residual,
+                                    uint16_t* out, int32_t* dev_status, void* ws, size_t ws_bytes,
+                                    void* stream);
 
 /* Pre-norm of a residual layer stack (not part of the paper's method; the layer stack workload
  * needs it, see the stack recurrence x_{l+1} = x_l + MoE(norm(x_l))): out[t] = x[t] / sqrt(mean_h
@@ -203,12 +229,29 @@ moe_status alloc_l_solve(const double* S, int32_t L, int32_t K_orig, int64_t B, 
 
 /* Instrumentation (no counterpart in the paper): with profiling on, moe_layer_forward records
  * CUDA events at its stage boundaries; moe_profile_read waits for the last forward call and
- * returns the device time in milliseconds of its 6 stages: gate, alloc_t_select, moe_permute,
- * expert GEMM-1 (with SwiGLU), expert GEMM-2, combine.  Host-side state only (events); one
- * forward call at a time may be in flight while profiling.  Off by default. */
+ * returns the device time in milliseconds of its 6 stages: gate; route (Alloc-T selection and the
+ * permutation's lists in one launch; beyond 8192 tokens the selection alone); gather (the copy of
+ * the routed rows, absent where the expert GEMM reads x by index; beyond 8192 tokens also the
+ * permutation's lists); expert GEMM-1 (with SwiGLU); expert GEMM-2; combine.  Host-side state only
+ * (events); one forward call at a time may be in flight while profiling.  Off by default. */
 #define MOE_PROFILE_STAGES 6
 moe_status moe_profile_enable(int32_t on);
 moe_status moe_profile_read(float* stage_ms /* host [MOE_PROFILE_STAGES] */);
+
+/* Self-test of the failure path (no counterpart in the paper).  Every device-side wait of the expert
+ * GEMMs is bounded: a wait that outlasts its limit raises MOE_ERR_TIMEOUT in dev_status, the CTA's other
+ * roles leave their loops at their next poll, the CTA waits for its copies in flight, frees its tensor
+ * memory and returns.  In production the limit is about half a second and nothing reaches it.  This
+ * call makes it happen on purpose, harmlessly: it launches expert GEMM-2 alone, with the row-block
+ * counters that GEMM-1 would fill cleared and never filled, and with the waits' limit set to
+ * wait_limit_clk SM clocks (1000 .. 2e9).  Expected outcome: the call returns MOE_OK, the kernel ends
+ * within a few multiples of the limit, dev_status holds 1 << MOE_ERR_TIMEOUT, y_perm is not written,
+ * and the next ordinary call on the same workspace is correct.
+ *   expert_offsets device int32 [N+1]; budget = rows of y_perm; W2 device bf16 [N,H,I];
+ *   y_perm device bf16 [budget,H]; ws as for moe_grouped_ffn */
+moe_status moe_selftest_wait_timeout(const moe_shape* shape, const int32_t* expert_offsets, int64_t budget,
+                                     const uint16_t* W2, uint16_t* y_perm, int64_t wait_limit_clk,
+                                     int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
 
 #ifdef __cplusplus
 }

@@ -61,8 +61,8 @@ def softmax_scores(logits) -> np.ndarray:
 
 
 def topk_sorted(scores, K_orig: int) -> Tuple[np.ndarray, np.ndarray]:
-    """Per token the K_orig largest scores, descending (Sec. 3.3: rows "sorted in
-    descending order"); equal scores rank the lower expert id first.
+    """Per token the K_orig largest scores, rows descending (the order Sec. 3.3's
+    procedure assumes); equal scores rank the lower expert id first.
     Returns (topk_idx int32 [T,K_orig], topk_score fp32 [T,K_orig])."""
     s = np.asarray(scores, np.float32)
     T, N = s.shape

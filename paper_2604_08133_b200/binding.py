@@ -16,8 +16,9 @@ MOE_OK, MOE_ERR_ARG, MOE_ERR_BUDGET, MOE_ERR_WORKSPACE, MOE_ERR_CUDA, MOE_ERR_NO
 
 EXPORTS = ("moe_status_string", "moe_workspace_bytes", "moe_gate", "alloc_t_select", "moe_permute",
            "moe_grouped_ffn", "moe_shared_ffn", "moe_combine", "moe_layer_forward", "moe_layer_intermediates",
-           "moe_rmsnorm", "moe_profile_enable", "moe_profile_read", "moe_permute_static", "moe_route", "alloc_l_solve")
-PROFILE_STAGES = ("gate", "select", "permute", "ffn_gemm1", "ffn_gemm2", "combine")
+           "moe_rmsnorm", "moe_profile_enable", "moe_profile_read", "moe_permute_static", "moe_route", "alloc_l_solve",
+           "moe_layer_forward_routed", "moe_selftest_wait_timeout")
+PROFILE_STAGES = ("gate", "route", "gather", "ffn_gemm1", "ffn_gemm2", "combine")
 
 
 class MoeShape(ctypes.Structure):
@@ -55,7 +56,9 @@ def lib() -> ctypes.CDLL:
             "moe_permute": [sp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, sz, vp],
             "moe_permute_static": [sp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp],
             "moe_route": [sp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp],
-            "moe_grouped_ffn": [sp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp],
+            "moe_grouped_ffn": [sp, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp],
+            "moe_layer_forward_routed": [sp, vp, vp, vp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp],
+            "moe_selftest_wait_timeout": [sp, vp, i64, vp, vp, i64, vp, vp, sz, vp],
             "moe_shared_ffn": [sp, vp, vp, vp, vp, vp, vp, sz, vp],
             "moe_combine": [sp, vp, vp, vp, vp, vp, vp, vp],
             "moe_layer_forward": [sp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, sz, vp],
@@ -164,10 +167,11 @@ def moe_permute_static(shape, x, topk_idx, topk_score, n_sel, budget, expert_off
                                                           _stream(stream)))
 
 
-def moe_grouped_ffn(shape, x_perm, expert_offsets, budget, W13, W2, y_perm, dev_status, ws, stream=None):
-    _check("moe_grouped_ffn", lib().moe_grouped_ffn(ctypes.byref(shape), _p(x_perm), _p(expert_offsets), int(budget),
-                                                    _p(W13), _p(W2), _p(y_perm), _p(dev_status), _p(ws), ws.numel(),
-                                                    _stream(stream)))
+def moe_grouped_ffn(shape, x_or_xperm, perm_token, expert_offsets, budget, W13, W2, y_perm, dev_status, ws, stream=None):
+    """perm_token None: x_or_xperm is x_perm [budget,H]; else it is x [T,H] and row p is x[perm_token[p]]."""
+    _check("moe_grouped_ffn", lib().moe_grouped_ffn(ctypes.byref(shape), _p(x_or_xperm), _p(perm_token),
+                                                    _p(expert_offsets), int(budget), _p(W13), _p(W2), _p(y_perm),
+                                                    _p(dev_status), _p(ws), ws.numel(), _stream(stream)))
 
 
 def moe_shared_ffn(shape, x, Wsh13, Wsh2, y_shared, dev_status, ws, stream=None):
@@ -185,6 +189,22 @@ def moe_layer_forward(shape, x, W_gate, gate_bias, W13, W2, Wsh13, Wsh2, budget,
     _check("moe_layer_forward", lib().moe_layer_forward(ctypes.byref(shape), _p(x), _p(W_gate), _p(gate_bias), _p(W13),
                                                         _p(W2), _p(Wsh13), _p(Wsh2), int(budget), _p(residual),
                                                         _p(out), _p(dev_status), _p(ws), ws.numel(), _stream(stream)))
+
+
+def moe_layer_forward_routed(shape, x, topk_idx, topk_score, n_sel, budget_max, budget_hint, W13, W2, Wsh13, Wsh2, out,
+                             dev_status, ws, residual: Optional[torch.Tensor] = None, stream=None):
+    """Permutation, experts and combine for a selection the caller holds (n_sel on the device)."""
+    _check("moe_layer_forward_routed",
+           lib().moe_layer_forward_routed(ctypes.byref(shape), _p(x), _p(topk_idx), _p(topk_score), _p(n_sel),
+                                          int(budget_max), int(budget_hint), _p(W13), _p(W2), _p(Wsh13), _p(Wsh2),
+                                          _p(residual), _p(out), _p(dev_status), _p(ws), ws.numel(), _stream(stream)))
+
+
+def moe_selftest_wait_timeout(shape, expert_offsets, budget, W2, y_perm, wait_limit_clk, dev_status, ws, stream=None):
+    """Launches expert GEMM-2 alone with a short wait limit: its bounded waits run out (see the header)."""
+    _check("moe_selftest_wait_timeout",
+           lib().moe_selftest_wait_timeout(ctypes.byref(shape), _p(expert_offsets), int(budget), _p(W2), _p(y_perm),
+                                           int(wait_limit_clk), _p(dev_status), _p(ws), ws.numel(), _stream(stream)))
 
 
 def moe_rmsnorm(shape, x, out, stream=None):

@@ -4,39 +4,28 @@
 
 #include "allocmoe.h"
 
+#include "ffn.h"
+#include "shape_check.h"
+
 // launchers defined next to their kernels
 moe_status launch_moe_gate(const moe_shape*, const uint16_t*, const uint16_t*, const float*, float*, int32_t*, float*,
                            int32_t*, int, cudaStream_t);
 moe_status launch_alloc_t_select(const moe_shape*, const float*, int64_t, int32_t*, int32_t*, cudaStream_t);
 moe_status launch_moe_permute(const moe_shape*, const uint16_t*, const int32_t*, const float*, const int32_t*, int64_t,
-                              int32_t*, int32_t*, float*, int32_t*, uint16_t*, int32_t*, int32_t*, cudaStream_t);
-moe_status launch_gather_rows(const moe_shape*, const uint16_t*, const int32_t*, int64_t, uint16_t*, cudaStream_t);
+                              int32_t*, int32_t*, float*, int32_t*, uint16_t*, int32_t*, int32_t*, bool, cudaStream_t);
+moe_status launch_gather_rows(const moe_shape*, const uint16_t*, const int32_t*, int64_t, const int32_t*, uint16_t*,
+                              cudaStream_t);
 bool moe_route_fits(const moe_shape*);
-moe_status launch_moe_route(const moe_shape*, const float*, const int32_t*, int64_t, int32_t*, int32_t*, int32_t*, float*,
-                            int32_t*, int32_t*, cudaStream_t);
-moe_status launch_ffn(const moe_shape*, const uint16_t*, const int32_t*, const int32_t*, int64_t, const uint16_t*, const uint16_t*,
-                      uint16_t*, uint16_t*, const uint16_t*, const uint16_t*, const uint16_t*, uint16_t*, uint16_t*,
-                      int32_t*, int32_t*, bool, cudaStream_t, cudaEvent_t);
-size_t ffn_done_ints(const moe_shape*, int64_t);
-bool ffn_gathers(const moe_shape*, int64_t);
+moe_status launch_moe_route(const moe_shape*, const float*, const int32_t*, int64_t, bool, int32_t*, int32_t*, int32_t*,
+                            float*, int32_t*, int32_t*, cudaStream_t);
 moe_status launch_moe_combine(const moe_shape*, const uint16_t*, const int32_t*, const float*, const int32_t*,
                               const uint16_t*, const uint16_t*, long long, uint16_t*, cudaStream_t);
 moe_status launch_rmsnorm(const moe_shape*, const uint16_t*, uint16_t*, cudaStream_t);
 
 namespace {
 
-bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
-bool shape_ok(const moe_shape* s) {
-  if (s == nullptr) return false;
-  if (s->flags != 0) return false;
-  if (s->T < 1 || s->H < 64 || s->I < 64 || s->N < 8 || s->S < 0) return false;
-  if (s->H % 64 != 0 || s->I % 64 != 0 || s->N % 4 != 0 || s->N > 128) return false;
-  if (s->K_orig < 1 || s->K_orig > 16 || s->K_orig > s->N) return false;
-  if (s->K_base < 0 || s->K_base > s->K_orig) return false;
-  if ((long long)s->T * s->K_orig >= (1ll << 31)) return false;
-  return true;
-}
+using allocmoe::aligned16;
+using allocmoe::shape_ok;
 
 bool budget_ok(const moe_shape* s, int64_t budget) {
   return budget >= (int64_t)s->K_base * s->T && budget <= (int64_t)s->K_orig * s->T;
@@ -79,7 +68,7 @@ template <typename T>
 T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<unsigned char*>(ws) + off); }
 
 // Optional stage timing of moe_layer_forward (off by default): events at the stage boundaries.
-constexpr int kProfStages = 6;   // gate, select, permute, ffn GEMM-1, ffn GEMM-2, combine
+constexpr int kProfStages = 6;   // gate, route, gather, ffn GEMM-1, ffn GEMM-2, combine
 bool g_prof_on = false;
 cudaEvent_t g_prof_ev[kProfStages + 1];
 void prof_mark(int i, cudaStream_t st) {
@@ -138,7 +127,7 @@ moe_status moe_permute(const moe_shape* shape, const uint16_t* x, const int32_t*
   const WsLayout L = ws_layout(shape, budget);
   if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
   return launch_moe_permute(shape, x, topk_idx, topk_score, n_sel, budget, expert_offsets, perm_token, perm_weight,
-                            pair_pos, x_perm, dev_status, at<int32_t>(ws, L.seg_counts), (cudaStream_t)stream);
+                            pair_pos, x_perm, dev_status, at<int32_t>(ws, L.seg_counts), true, (cudaStream_t)stream);
 }
 
 moe_status moe_route(const moe_shape* shape, const int32_t* topk_idx, const float* topk_score, int64_t budget,
@@ -150,20 +139,43 @@ moe_status moe_route(const moe_shape* shape, const int32_t* topk_idx, const floa
   if (!aligned16(topk_idx) || !aligned16(topk_score) || !aligned16(n_sel)) return MOE_ERR_ARG;
   if (!moe_route_fits(shape)) return MOE_ERR_ARG;
   if (!budget_ok(shape, budget)) return MOE_ERR_BUDGET;
-  return launch_moe_route(shape, topk_score, topk_idx, budget, n_sel, expert_offsets, perm_token, perm_weight, pair_pos,
-                          dev_status, (cudaStream_t)stream);
+  return launch_moe_route(shape, topk_score, topk_idx, budget, false, n_sel, expert_offsets, perm_token, perm_weight,
+                          pair_pos, dev_status, (cudaStream_t)stream);
 }
 
-moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_perm, const int32_t* expert_offsets,
-                           int64_t budget, const uint16_t* W13, const uint16_t* W2, uint16_t* y_perm,
-                           int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
-  if (!shape_ok(shape) || !x_perm || !expert_offsets || !W13 || !W2 || !y_perm || !dev_status || !ws) return MOE_ERR_ARG;
-  if (!aligned16(x_perm) || !aligned16(W13) || !aligned16(W2) || !aligned16(y_perm) || !aligned16(ws)) return MOE_ERR_ARG;
+moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_or_xperm, const int32_t* perm_token,
+                           const int32_t* expert_offsets, int64_t budget, const uint16_t* W13, const uint16_t* W2,
+                           uint16_t* y_perm, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  if (!shape_ok(shape) || !x_or_xperm || !expert_offsets || !W13 || !W2 || !y_perm || !dev_status || !ws)
+    return MOE_ERR_ARG;
+  if (!aligned16(x_or_xperm) || !aligned16(W13) || !aligned16(W2) || !aligned16(y_perm) || !aligned16(ws))
+    return MOE_ERR_ARG;
   if (budget < 0 || budget > (int64_t)shape->K_orig * shape->T) return MOE_ERR_BUDGET;
   const WsLayout L = ws_layout(shape, budget);
   if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
-  return launch_ffn(shape, x_perm, nullptr, expert_offsets, budget, W13, W2, at<uint16_t>(ws, L.h), y_perm, nullptr, nullptr,
-                    nullptr, nullptr, nullptr, dev_status, at<int32_t>(ws, L.gemm_done), false, (cudaStream_t)stream, nullptr);
+  cudaStream_t st = (cudaStream_t)stream;
+  FfnArgs a;
+  a.s = shape;
+  a.a_routed = x_or_xperm;
+  a.gather_idx = perm_token;
+  if (perm_token != nullptr && budget > 0 && !ffn_gathers(shape, budget)) {
+    // long expert runs: one copy of the rows into the workspace, then 128-row box loads, is faster than
+    // fetching every tile's rows four at a time
+    const moe_status r = launch_gather_rows(shape, x_or_xperm, perm_token, budget, nullptr, at<uint16_t>(ws, L.x_perm), st);
+    if (r != MOE_OK) return r;
+    a.a_routed = at<uint16_t>(ws, L.x_perm);
+    a.gather_idx = nullptr;
+  }
+  a.expert_offsets = expert_offsets;
+  a.budget = budget;
+  a.W13 = W13;
+  a.W2 = W2;
+  a.h = at<uint16_t>(ws, L.h);
+  a.y_perm = y_perm;
+  a.dev_status = dev_status;
+  a.done = at<int32_t>(ws, L.gemm_done);
+  a.stream = st;
+  return launch_ffn(a);
 }
 
 moe_status moe_shared_ffn(const moe_shape* shape, const uint16_t* x, const uint16_t* Wsh13, const uint16_t* Wsh2,
@@ -172,9 +184,17 @@ moe_status moe_shared_ffn(const moe_shape* shape, const uint16_t* x, const uint1
   if (!aligned16(x) || !aligned16(Wsh13) || !aligned16(Wsh2) || !aligned16(y_shared) || !aligned16(ws)) return MOE_ERR_ARG;
   const WsLayout L = ws_layout(shape, 0);
   if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
-  return launch_ffn(shape, nullptr, nullptr, nullptr, 0, nullptr, nullptr, nullptr, nullptr, x, Wsh13, Wsh2,
-                    at<uint16_t>(ws, L.h_sh), y_shared, dev_status, at<int32_t>(ws, L.gemm_done), false,
-                    (cudaStream_t)stream, nullptr);
+  FfnArgs a;
+  a.s = shape;
+  a.x_shared = x;
+  a.Wsh13 = Wsh13;
+  a.Wsh2 = Wsh2;
+  a.h_sh = at<uint16_t>(ws, L.h_sh);
+  a.y_shared = y_shared;
+  a.dev_status = dev_status;
+  a.done = at<int32_t>(ws, L.gemm_done);
+  a.stream = (cudaStream_t)stream;
+  return launch_ffn(a);
 }
 
 moe_status moe_combine(const moe_shape* shape, const uint16_t* y_perm, const int32_t* pair_pos,
@@ -222,30 +242,138 @@ moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const ui
   prof_mark(1, st);
   if (moe_route_fits(shape)) {
     // selection and permutation bookkeeping in one launch, then the row gather
-    r = launch_moe_route(shape, topk_score, topk_idx, budget, n_sel, expert_offsets, perm_token, perm_weight, pair_pos,
-                         dev_status, st);
+    r = launch_moe_route(shape, topk_score, topk_idx, budget, false, n_sel, expert_offsets, perm_token, perm_weight,
+                         pair_pos, dev_status, st);
     if (r != MOE_OK) return r;
     prof_mark(2, st);
-    if (budget > 0 && x_perm != nullptr) r = launch_gather_rows(shape, x, perm_token, budget, x_perm, st);
+    if (budget > 0 && x_perm != nullptr) r = launch_gather_rows(shape, x, perm_token, budget, nullptr, x_perm, st);
   } else {
     r = launch_alloc_t_select(shape, topk_score, budget, n_sel, dev_status, st);
     if (r != MOE_OK) return r;
     prof_mark(2, st);
     r = launch_moe_permute(shape, x, topk_idx, topk_score, n_sel, budget, expert_offsets, perm_token, perm_weight,
-                           pair_pos, x_perm, dev_status, at<int32_t>(ws, L.seg_counts), st);
+                           pair_pos, x_perm, dev_status, at<int32_t>(ws, L.seg_counts), true, st);
   }
   if (r != MOE_OK) return r;
   prof_mark(3, st);
-  r = launch_ffn(shape, x_perm != nullptr ? x_perm : x, x_perm != nullptr ? nullptr : perm_token, expert_offsets, budget,
-                 W13, W2, at<uint16_t>(ws, L.h), y_perm,
-                 shape->S > 0 ? x : nullptr, Wsh13, Wsh2, at<uint16_t>(ws, L.h_sh), y_shared, dev_status,
-                 at<int32_t>(ws, L.gemm_done), true, st, g_prof_on ? g_prof_ev[4] : nullptr);
+  FfnArgs a;
+  a.s = shape;
+  a.a_routed = x_perm != nullptr ? x_perm : x;
+  a.gather_idx = x_perm != nullptr ? nullptr : perm_token;
+  a.expert_offsets = expert_offsets;
+  a.budget = budget;
+  a.W13 = W13;
+  a.W2 = W2;
+  a.h = at<uint16_t>(ws, L.h);
+  a.y_perm = y_perm;
+  a.x_shared = shape->S > 0 ? x : nullptr;
+  a.Wsh13 = Wsh13;
+  a.Wsh2 = Wsh2;
+  a.h_sh = at<uint16_t>(ws, L.h_sh);
+  a.y_shared = y_shared;
+  a.dev_status = dev_status;
+  a.done = at<int32_t>(ws, L.gemm_done);
+  a.done_is_clear = true;
+  a.stream = st;
+  a.between = g_prof_on ? g_prof_ev[4] : nullptr;
+  r = launch_ffn(a);
   if (r != MOE_OK) return r;
   prof_mark(5, st);
   r = launch_moe_combine(shape, y_perm, pair_pos, topk_score, n_sel, y_shared, residual, budget, out,
                          st);
   prof_mark(6, st);
   return r;
+}
+
+moe_status moe_layer_forward_routed(const moe_shape* shape, const uint16_t* x, const int32_t* topk_idx,
+                                    const float* topk_score, const int32_t* n_sel, int64_t budget_max,
+                                    int64_t budget_hint, const uint16_t* W13, const uint16_t* W2, const uint16_t* Wsh13,
+                                    const uint16_t* Wsh2, const uint16_t* residual, uint16_t* out, int32_t* dev_status,
+                                    void* ws, size_t ws_bytes, void* stream) {
+  if (!shape_ok(shape) || !x || !topk_idx || !topk_score || !n_sel || !W13 || !W2 || !out || !dev_status || !ws)
+    return MOE_ERR_ARG;
+  if (shape->S > 0 && (!Wsh13 || !Wsh2)) return MOE_ERR_ARG;
+  // n_sel is read one int at a time: a slice of a longer array (this rank's part of the pool's counts) is fine
+  if (!aligned16(x) || !aligned16(topk_idx) || !aligned16(topk_score) || !aligned16(W13) || !aligned16(W2) ||
+      !aligned16(out) || !aligned16(ws) || (reinterpret_cast<uintptr_t>(n_sel) & 3u) != 0)
+    return MOE_ERR_ARG;
+  if (shape->S > 0 && (!aligned16(Wsh13) || !aligned16(Wsh2))) return MOE_ERR_ARG;
+  if (residual != nullptr && (!aligned16(residual) || residual == out)) return MOE_ERR_ARG;
+  if (budget_max < 0 || budget_max > (int64_t)shape->K_orig * shape->T) return MOE_ERR_BUDGET;
+  if (budget_hint < 0) return MOE_ERR_BUDGET;
+  const WsLayout L = ws_layout(shape, budget_max);
+  if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int64_t expected = (budget_hint > 0 && budget_hint < budget_max) ? budget_hint : budget_max;
+  int32_t* expert_offsets = at<int32_t>(ws, L.expert_offsets);
+  int32_t* perm_token = at<int32_t>(ws, L.perm_token);
+  float* perm_weight = at<float>(ws, L.perm_weight);
+  int32_t* pair_pos = at<int32_t>(ws, L.pair_pos);
+  uint16_t* x_perm = at<uint16_t>(ws, L.x_perm);
+  uint16_t* y_perm = at<uint16_t>(ws, L.y_perm);
+  uint16_t* y_shared = shape->S > 0 ? at<uint16_t>(ws, L.y_shared) : nullptr;
+  if (ffn_gathers(shape, expected)) x_perm = nullptr;
+
+  moe_status r;
+  if (moe_route_fits(shape)) {
+    r = launch_moe_route(shape, topk_score, topk_idx, budget_max, true, const_cast<int32_t*>(n_sel), expert_offsets,
+                         perm_token, perm_weight, pair_pos, dev_status, st);
+    if (r != MOE_OK) return r;
+    if (budget_max > 0 && x_perm != nullptr)
+      r = launch_gather_rows(shape, x, perm_token, budget_max, expert_offsets + shape->N, x_perm, st);
+  } else {
+    r = launch_moe_permute(shape, x, topk_idx, topk_score, n_sel, budget_max, expert_offsets, perm_token, perm_weight,
+                           pair_pos, x_perm, dev_status, at<int32_t>(ws, L.seg_counts), false, st);
+  }
+  if (r != MOE_OK) return r;
+  FfnArgs a;
+  a.s = shape;
+  a.a_routed = x_perm != nullptr ? x_perm : x;
+  a.gather_idx = x_perm != nullptr ? nullptr : perm_token;
+  a.expert_offsets = expert_offsets;
+  a.budget = budget_max;
+  a.budget_hint = expected;
+  a.W13 = W13;
+  a.W2 = W2;
+  a.h = at<uint16_t>(ws, L.h);
+  a.y_perm = y_perm;
+  a.x_shared = shape->S > 0 ? x : nullptr;
+  a.Wsh13 = Wsh13;
+  a.Wsh2 = Wsh2;
+  a.h_sh = at<uint16_t>(ws, L.h_sh);
+  a.y_shared = y_shared;
+  a.dev_status = dev_status;
+  a.done = at<int32_t>(ws, L.gemm_done);
+  a.stream = st;
+  r = launch_ffn(a);
+  if (r != MOE_OK) return r;
+  return launch_moe_combine(shape, y_perm, pair_pos, topk_score, n_sel, y_shared, residual, budget_max, out, st);
+}
+
+moe_status moe_selftest_wait_timeout(const moe_shape* shape, const int32_t* expert_offsets, int64_t budget,
+                                     const uint16_t* W2, uint16_t* y_perm, int64_t wait_limit_clk, int32_t* dev_status,
+                                     void* ws, size_t ws_bytes, void* stream) {
+  if (!shape_ok(shape) || !expert_offsets || !W2 || !y_perm || !dev_status || !ws) return MOE_ERR_ARG;
+  if (!aligned16(W2) || !aligned16(y_perm) || !aligned16(ws)) return MOE_ERR_ARG;
+  if (budget < 1 || budget > (int64_t)shape->K_orig * shape->T) return MOE_ERR_BUDGET;
+  if (wait_limit_clk < 1000 || wait_limit_clk > 2000000000ll) return MOE_ERR_ARG;
+  const WsLayout L = ws_layout(shape, budget);
+  if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
+  FfnArgs a;
+  a.s = shape;
+  a.a_routed = at<uint16_t>(ws, L.x_perm);   // never read: GEMM-1 is not launched
+  a.expert_offsets = expert_offsets;
+  a.budget = budget;
+  a.W13 = W2;                                 // only a tensor map is built from it
+  a.W2 = W2;
+  a.h = at<uint16_t>(ws, L.h);
+  a.y_perm = y_perm;
+  a.dev_status = dev_status;
+  a.done = at<int32_t>(ws, L.gemm_done);      // cleared by launch_ffn, then never incremented
+  a.wait_limit_clk = wait_limit_clk;
+  a.gemm2_only = true;
+  a.stream = (cudaStream_t)stream;
+  return launch_ffn(a);
 }
 
 moe_status moe_rmsnorm(const moe_shape* shape, const uint16_t* x, uint16_t* out, void* stream) {

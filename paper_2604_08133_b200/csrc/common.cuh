@@ -7,6 +7,7 @@
 #include <stdint.h>
 
 #include "allocmoe.h"
+#include "device_once.h"
 
 #define DEV __device__ __forceinline__
 
@@ -30,7 +31,10 @@ DEV void pdl_prologue_done() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
-constexpr long long kWaitLimitClk = 1000ll * 1000ll * 1000ll;   // bounded waits: about 0.5 s at 1.9 GHz
+// Default limit of the bounded waits below, in SM clocks: about 0.5 s at 1.9 GHz.  Kernels take the
+// limit as a launch parameter (FfnGemmParams::wait_limit_clk) so that a test can make a wait run out
+// within milliseconds; every product launch passes this value.
+constexpr long long kWaitLimitClk = 1000ll * 1000ll * 1000ll;
 DEV void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 DEV void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -50,7 +54,8 @@ DEV int flag_load_acquire(const int32_t* flag) {
   return v;
 }
 // Bounded wait for *flag >= need (same limit and abort protocol as the mbarrier waits).
-DEV bool flag_wait_bounded(const int32_t* flag, int need, volatile int* abort_flag, int32_t* dev_status) {
+DEV bool flag_wait_bounded(const int32_t* flag, int need, volatile int* abort_flag, int32_t* dev_status,
+                           long long limit_clk) {
   if (flag_load_acquire(flag) >= need) return true;
   long long t0 = 0;
   uint32_t spins = 0;
@@ -62,7 +67,7 @@ DEV bool flag_wait_bounded(const int32_t* flag, int need, volatile int* abort_fl
       const long long now = clock64();
       if (t0 == 0) {
         t0 = now;
-      } else if (now - t0 > kWaitLimitClk) {
+      } else if (now - t0 > limit_clk) {
         *abort_flag = 1;
         set_dev_status(dev_status, MOE_ERR_TIMEOUT);
         return false;
@@ -93,14 +98,15 @@ DEV bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Every wait in these kernels is bounded.  A wait that exceeds kWaitLimitClk raises the CTA's
+// Every wait in these kernels is bounded.  A wait that exceeds its limit (limit_clk) raises the CTA's
 // abort flag and MOE_ERR_TIMEOUT in the caller's status word; every other wait of the CTA
 // then returns false at its next poll, the roles leave their loops and the CTA tears down
 // normally (drains its own copies, frees TMEM, returns).  Time is the SM's own cycle counter,
 // looked at only every 64th poll, so a wait that succeeds quickly never pays for it.
 constexpr long long kDrainLimitClk = 40ll * 1000ll * 1000ll;    // teardown waits: about 20 ms
 
-DEV bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
+DEV bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status,
+                           long long limit_clk) {
   if (mbar_try_wait(bar, parity)) return true;
   long long t0 = 0;
   uint32_t spins = 0;
@@ -111,7 +117,7 @@ DEV bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_f
       const long long now = clock64();
       if (t0 == 0) {
         t0 = now;
-      } else if (now - t0 > kWaitLimitClk) {
+      } else if (now - t0 > limit_clk) {
         *abort_flag = 1;
         set_dev_status(dev_status, MOE_ERR_TIMEOUT);
         return false;
@@ -123,7 +129,8 @@ DEV bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_f
 // The same wait for a whole warp whose lanes all need the result: lane 0 polls, with a short
 // sleep between polls, and the outcome is broadcast, so that 128 epilogue threads do not all
 // poll the same barrier word.
-DEV bool mbar_wait_bounded_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
+DEV bool mbar_wait_bounded_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status,
+                                long long limit_clk) {
   int ok = 1;
   if ((threadIdx.x & 31) == 0) {
     if (!mbar_try_wait(bar, parity)) {
@@ -137,7 +144,7 @@ DEV bool mbar_wait_bounded_warp(uint64_t* bar, uint32_t parity, volatile int* ab
           const long long now = clock64();
           if (t0 == 0) {
             t0 = now;
-          } else if (now - t0 > kWaitLimitClk) {
+          } else if (now - t0 > limit_clk) {
             *abort_flag = 1;
             set_dev_status(dev_status, MOE_ERR_TIMEOUT);
             ok = 0;
@@ -373,6 +380,18 @@ DEV int block_exclusive_scan(int v, int* warp_sums, int* total) {
 }
 
 }  // namespace allocmoe
+
+// Host side.  Lets `kernel` use `bytes` of dynamic shared memory on the current device; the attribute is
+// per device, so `once` remembers the devices it has been set on.
+template <typename Kernel>
+inline bool ensure_dynamic_smem(Kernel kernel, size_t bytes, allocmoe::PerDeviceOnce& once) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  if (once.done(dev)) return true;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return false;
+  once.mark(dev);
+  return true;
+}
 
 // Host side: launch with the programmatic-stream-serialization attribute (and, when cluster_y > 1,
 // a thread-block cluster).

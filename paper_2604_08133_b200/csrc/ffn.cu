@@ -1,6 +1,6 @@
 // Grouped SwiGLU expert GEMMs on the 5th-generation tensor cores (tcgen05 + TMEM), fed by TMA.
 //
-// "Each activated expert corresponds to one feed-forward execution" (Sec. 3.1): for the rows of
+// One expert feed-forward execution per kept (token, expert) pair (Sec. 3.1): for the rows of
 // expert e (a contiguous run of the permuted list)
 //     GEMM-1   h = silu(X W1_e^T) * (X W3_e^T)       [rows, I]   (SwiGLU fused in the epilogue)
 //     GEMM-2   y = h W2_e^T                          [rows, H]
@@ -31,6 +31,7 @@
 #include <stdlib.h>
 
 #include "common.cuh"
+#include "ffn.h"
 
 namespace allocmoe {
 
@@ -68,9 +69,13 @@ struct FfnGemmParams {
   // GEMM-2 may start while GEMM-1 is still running: per block of token rows, GEMM-1 counts the tiles
   // of h it has finished (done[block], once per epilogue warp) and GEMM-2 loads a block's rows once
   // the count reaches dep_need_* (GEMM-1's tiles per block x epilogue warps).  nullptr = no tracking.
+  // Invariant: a GEMM-2 launch that was handed `done` does not complete before the GEMM-1 launch ahead of it
+  // in the stream has (it executes griddepcontrol.wait in its teardown at the latest, also when a bounded
+  // wait gave up), so whatever follows GEMM-2 in the stream may reuse h, `done` and the workspace.
   int32_t* done;
   int done_capacity;                // counters behind `done`; offsets that need more (inconsistent input) switch tracking off
   int dep_need_routed, dep_need_shared;
+  long long wait_limit_clk;         // limit of every bounded wait of the launch, in SM clocks (kWaitLimitClk)
   // gather_rows > 0: the routed A tensor map has a box one row high and the producer warp fetches a
   // tile's rows four per TMA instruction, only those that hold rows of the expert's run.  GEMM-1 can
   // then read the routed tokens' rows straight from x instead of a permuted copy: row m of the routed
@@ -309,7 +314,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
         if (!kSwiGLU && track) {   // the block's rows of h are complete?
           if (lane == 0)
             ok = flag_wait_bounded(p.done + tc.dep_id, tc.shared ? p.dep_need_shared : p.dep_need_routed, abort_flag,
-                                   p.dev_status);
+                                   p.dev_status, p.wait_limit_clk);
           if (gather) {
             __syncwarp();
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -320,8 +325,8 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          ok = gather ? mbar_wait_bounded_warp(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status)
-                      : mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status);
+          ok = gather ? mbar_wait_bounded_warp(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status, p.wait_limit_clk)
+                      : mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status, p.wait_limit_clk);
           if (!ok) break;
           unsigned char* sa = tiles + s * kStageBytes;
           unsigned char* sb = sa + kABytes;
@@ -363,13 +368,13 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
         const TileCoord tc = w.at(tile, p);
         const int nkb = tc.shared ? kb_shared : kb_routed;
         const uint32_t a = tcount & 1u, aph = (tcount >> 1) & 1u;
-        if (!(ok = mbar_wait_bounded(&ctl->tmem_empty[a], aph ^ 1u, abort_flag, p.dev_status))) break;
+        if (!(ok = mbar_wait_bounded(&ctl->tmem_empty[a], aph ^ 1u, abort_flag, p.dev_status, p.wait_limit_clk))) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + a * kAccCols;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!(ok = mbar_wait_bounded(&ctl->full[s], ph, abort_flag, p.dev_status))) break;
+          if (!(ok = mbar_wait_bounded(&ctl->full[s], ph, abort_flag, p.dev_status, p.wait_limit_clk))) break;
           tc_fence_after_sync();
           const uint32_t sa = smem_u32(tiles + s * kStageBytes);
           const uint64_t da = umma_desc_sw128(sa), db = umma_desc_sw128(sa + kABytes);
@@ -395,7 +400,7 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
       if (tile >= total_tiles) break;
       const TileCoord tc = w.at(tile, p);
       const uint32_t a = tcount & 1u, aph = (tcount >> 1) & 1u;
-      if (!(ok = mbar_wait_bounded_warp(&ctl->tmem_full[a], aph, abort_flag, p.dev_status))) break;
+      if (!(ok = mbar_wait_bounded_warp(&ctl->tmem_full[a], aph, abort_flag, p.dev_status, p.wait_limit_clk))) break;
       tc_fence_after_sync();
       const int row = tc.m0 + q * 32 + lane;
       const bool row_ok = row < tc.m_end;
@@ -466,6 +471,10 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   }
 
   // ---------------- teardown
+  // GEMM-2 with row-block tracking has not waited for the whole of GEMM-1 yet.  It does so here, on the abort
+  // path too, so that its completion implies GEMM-1's (FfnGemmParams::done); in the normal case GEMM-1 has
+  // finished long before and the wait is free.
+  if (!kSwiGLU && p.done != nullptr) pdl_wait();
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) {
@@ -587,7 +596,7 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
         if (!kSwiGLU && track) {   // the block's rows of h are complete?
           if (lane == 0)
             ok = flag_wait_bounded(p.done + tc.dep_id, tc.shared ? p.dep_need_shared : p.dep_need_routed, abort_flag,
-                                   p.dev_status);
+                                   p.dev_status, p.wait_limit_clk);
           if (gather) {
             __syncwarp();
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -598,8 +607,8 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % kPairStages;
           const uint32_t ph = (it / kPairStages) & 1u;
-          ok = gather ? mbar_wait_bounded_warp(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status)
-                      : mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status);
+          ok = gather ? mbar_wait_bounded_warp(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status, p.wait_limit_clk)
+                      : mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag, p.dev_status, p.wait_limit_clk);
           if (!ok) break;
           unsigned char* sa = tiles + s * kPairStageBytes;
           unsigned char* sb = sa + kABytes;
@@ -643,13 +652,13 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
         const TileCoord tc = w.at(tile, p);
         const int nkb = tc.shared ? kb_shared : kb_routed;
         const uint32_t a = tcount & 1u, aph = (tcount >> 1) & 1u;
-        if (!(ok = mbar_wait_bounded(&ctl->tmem_empty[a], aph ^ 1u, abort_flag, p.dev_status))) break;
+        if (!(ok = mbar_wait_bounded(&ctl->tmem_empty[a], aph ^ 1u, abort_flag, p.dev_status, p.wait_limit_clk))) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + a * kAccCols;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % kPairStages;
           const uint32_t ph = (it / kPairStages) & 1u;
-          if (!(ok = mbar_wait_bounded(&ctl->full[s], ph, abort_flag, p.dev_status))) break;
+          if (!(ok = mbar_wait_bounded(&ctl->full[s], ph, abort_flag, p.dev_status, p.wait_limit_clk))) break;
           tc_fence_after_sync();
           const uint32_t sa = smem_u32(tiles + s * kPairStageBytes);
           const uint64_t da = umma_desc_sw128(sa), db = umma_desc_sw128(sa + kABytes);
@@ -675,7 +684,7 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
       if (tile >= total_tiles) break;
       const TileCoord tc = w.at(tile, p);
       const uint32_t a = tcount & 1u, aph = (tcount >> 1) & 1u;
-      if (!(ok = mbar_wait_bounded_warp(&ctl->tmem_full[a], aph, abort_flag, p.dev_status))) break;
+      if (!(ok = mbar_wait_bounded_warp(&ctl->tmem_full[a], aph, abort_flag, p.dev_status, p.wait_limit_clk))) break;
       tc_fence_after_sync();
       const int row0 = tc.m0 + (int)rank * kBM + q * 32;
       const int row = row0 + lane;
@@ -745,6 +754,7 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
   }
 
   // ---------------- teardown: neither CTA leaves (or frees TMEM) while its peer may still touch it
+  if (!kSwiGLU && p.done != nullptr) pdl_wait();   // GEMM-2's completion implies GEMM-1's (see the one-CTA kernel)
   tc_fence_before_sync();
   __syncthreads();
   cluster_sync_all();
@@ -793,15 +803,17 @@ static bool make_tmap(CUtensorMap* tm, const void* base, uint64_t d0, uint64_t d
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static int g_num_sms = 0;
+// SM count of the current device (the persistent kernels' grid), looked up once per device.
+static PerDeviceInt g_num_sms;
 static int num_sms() {
-  if (g_num_sms == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
-    if (g_num_sms <= 0) g_num_sms = 148;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  int n = g_num_sms.get(dev);
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    g_num_sms.set(dev, n);
   }
-  return g_num_sms;
+  return n;
 }
 
 
@@ -810,13 +822,8 @@ static moe_status launch_gemm(const FfnGemmParams& p, const CUtensorMap& ar, con
                               const CUtensorMap& as, const CUtensorMap& bs, cudaStream_t stream) {
   constexpr size_t smem = TileCfg<kN>::kSmemBytes + sizeof(FfnSmemCtl) + 1024;
   static_assert(smem <= 232448, "ring + control block exceed the 227 KB a CTA may use");
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(ffn_gemm_kernel<kSwiGLU, kN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-        cudaSuccess)
-      return MOE_ERR_CUDA;
-    attr_done = true;
-  }
+  static PerDeviceOnce attr_set;
+  if (!ensure_dynamic_smem(ffn_gemm_kernel<kSwiGLU, kN>, smem, attr_set)) return MOE_ERR_CUDA;
   return launch_dependent(ffn_gemm_kernel<kSwiGLU, kN>, dim3((unsigned)num_sms()), dim3(kFfnThreads), smem, stream, 1, p,
                           ar, br, as, bs) == cudaSuccess
              ? MOE_OK
@@ -828,13 +835,8 @@ static moe_status launch_gemm_pair(const FfnGemmParams& p, const CUtensorMap& ar
                                    const CUtensorMap& as, const CUtensorMap& bs, cudaStream_t stream) {
   constexpr size_t smem = (size_t)kPairStages * kPairStageBytes + sizeof(FfnSmemCtl) + 1024;
   static_assert(smem <= 232448, "ring + control block exceed the 227 KB a CTA may use");
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(ffn_gemm_pair_kernel<kSwiGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-        cudaSuccess)
-      return MOE_ERR_CUDA;
-    attr_done = true;
-  }
+  static PerDeviceOnce attr_set;
+  if (!ensure_dynamic_smem(ffn_gemm_pair_kernel<kSwiGLU>, smem, attr_set)) return MOE_ERR_CUDA;
   const unsigned grid = (unsigned)(num_sms() & ~1);
   return launch_dependent_cluster(ffn_gemm_pair_kernel<kSwiGLU>, dim3(grid), dim3(kFfnThreads), smem, stream,
                                   dim3(2, 1, 1), p, ar, br, as, bs) == cudaSuccess
@@ -891,91 +893,94 @@ bool ffn_gathers(const moe_shape* s, int64_t budget) {
   return budget > 0 && budget <= (int64_t)limit * s->N;
 }
 
-// Routed and/or shared experts in one pair of launches.
-//   routed part present iff budget > 0 && x_perm != nullptr; shared part iff S > 0 && x_shared != nullptr.
-//   gather_idx != nullptr: x_perm is x [T, H] itself and routed row m is x[gather_idx[m]] (perm_token);
+// Routed and/or shared experts in one pair of launches (FfnArgs in ffn.h).
+//   routed part present iff budget > 0 && a_routed != nullptr; shared part iff S > 0 && x_shared != nullptr.
+//   gather_idx != nullptr: a_routed is x [T, H] itself and routed row m is x[gather_idx[m]] (perm_token);
 //   callers pass it only where ffn_gathers() holds.
 //   done_is_clear: an earlier kernel of the stream has zeroed `done` (else a memset is enqueued here).
-moe_status launch_ffn(const moe_shape* s, const uint16_t* x_perm, const int32_t* gather_idx,
-                      const int32_t* expert_offsets, int64_t budget,
-                      const uint16_t* W13, const uint16_t* W2, uint16_t* h, uint16_t* y_perm, const uint16_t* x_shared,
-                      const uint16_t* Wsh13, const uint16_t* Wsh2, uint16_t* h_sh, uint16_t* y_shared,
-                      int32_t* dev_status, int32_t* done, bool done_is_clear, cudaStream_t stream, cudaEvent_t between) {
-  const bool routed = (budget > 0 && x_perm != nullptr);
-  const bool shared = (s->S > 0 && x_shared != nullptr);
+moe_status launch_ffn(const FfnArgs& a) {
+  const moe_shape* s = a.s;
+  const int64_t budget = a.budget;
+  const bool routed = (budget > 0 && a.a_routed != nullptr);
+  const bool shared = (s->S > 0 && a.x_shared != nullptr);
   if (!routed && !shared) return MOE_OK;
+  const int64_t expected = !routed ? 0 : (a.budget_hint > 0 && a.budget_hint < budget ? a.budget_hint : budget);
   const uint64_t H = s->H, I = s->I;
   CUtensorMap a1r, b1r, a1s, b1s, a2r, b2r, a2s, b2s;
-  const bool pairs = use_pairs(s, routed ? budget : 0);
-  const int tile_n = pairs ? 256 : pick_tile_n(s, routed ? budget : 0, shared);
+  const bool pairs = use_pairs(s, expected);
+  const int tile_n = pairs ? 256 : pick_tile_n(s, expected, shared);
   const uint32_t kUmmaN = (uint32_t)tile_n;
   const uint32_t b2_box = pairs ? kUmmaN / 2 : kUmmaN;   // a pair's CTA loads half of the B tile
-  const bool by_rows = routed && (gather_idx != nullptr || ffn_gathers(s, budget));
+  const bool by_rows = routed && (a.gather_idx != nullptr || ffn_gathers(s, expected));
   bool ok = true;
   if (routed) {
-    if (gather_idx != nullptr) ok &= make_tmap(&a1r, x_perm, H, (uint64_t)s->T, 0, H, 0, 1);
-    else ok &= make_tmap(&a1r, x_perm, H, (uint64_t)budget, 0, H, 0, by_rows ? 1 : kBM);
-    ok &= make_tmap(&b1r, W13, H, 2 * I, (uint64_t)s->N, H, 2 * I * H, kUmmaN / 2);
-    ok &= make_tmap(&a2r, h, I, (uint64_t)budget, 0, I, 0, by_rows ? 1 : kBM);
-    ok &= make_tmap(&b2r, W2, I, H, (uint64_t)s->N, I, H * I, b2_box);
+    if (a.gather_idx != nullptr) ok &= make_tmap(&a1r, a.a_routed, H, (uint64_t)s->T, 0, H, 0, 1);
+    else ok &= make_tmap(&a1r, a.a_routed, H, (uint64_t)budget, 0, H, 0, by_rows ? 1 : kBM);
+    ok &= make_tmap(&b1r, a.W13, H, 2 * I, (uint64_t)s->N, H, 2 * I * H, kUmmaN / 2);
+    ok &= make_tmap(&a2r, a.h, I, (uint64_t)budget, 0, I, 0, by_rows ? 1 : kBM);
+    ok &= make_tmap(&b2r, a.W2, I, H, (uint64_t)s->N, I, H * I, b2_box);
   }
   if (shared) {
     const uint64_t S = s->S;
-    ok &= make_tmap(&a1s, x_shared, H, (uint64_t)s->T, 0, H, 0, kBM);
-    ok &= make_tmap(&b1s, Wsh13, H, 2 * I, S, H, 2 * I * H, kUmmaN / 2);
-    ok &= make_tmap(&a2s, h_sh, S * I, (uint64_t)s->T, 0, S * I, 0, kBM);
-    ok &= make_tmap(&b2s, Wsh2, I, H, S, I, H * I, b2_box);
+    ok &= make_tmap(&a1s, a.x_shared, H, (uint64_t)s->T, 0, H, 0, kBM);
+    ok &= make_tmap(&b1s, a.Wsh13, H, 2 * I, S, H, 2 * I * H, kUmmaN / 2);
+    ok &= make_tmap(&a2s, a.h_sh, S * I, (uint64_t)s->T, 0, S * I, 0, kBM);
+    ok &= make_tmap(&b2s, a.Wsh2, I, H, S, I, H * I, b2_box);
   }
   if (!ok) return MOE_ERR_CUDA;
   if (!routed) { a1r = a1s; b1r = b1s; a2r = a2s; b2r = b2s; }
   if (!shared) { a1s = a1r; b1s = b1r; a2s = a2r; b2s = b2r; }
 
   FfnGemmParams p{};
-  p.expert_offsets = expert_offsets;
+  p.expert_offsets = a.expert_offsets;
   p.n_experts = routed ? s->N : 0;
   p.routed_rows = routed ? (int)budget : 0;
   p.shared_rows = shared ? s->T : 0;
   p.shared_sub = s->S;
-  p.dev_status = dev_status;
+  p.dev_status = a.dev_status;
+  p.wait_limit_clk = a.wait_limit_clk > 0 ? a.wait_limit_clk : kWaitLimitClk;
   // row-block completion counters for the GEMM-1 -> GEMM-2 hand-over
-  p.done = done;
-  if (done != nullptr) {
+  p.done = a.done;
+  if (a.done != nullptr) {
     const int nb1 = (int)((s->I + kUmmaN / 2 - 1) / (kUmmaN / 2));      // GEMM-1 column blocks per (sub-)expert
     const int per_tile = 4 * (pairs ? 2 : 1);                           // every epilogue warp counts once
     p.dep_need_routed = nb1 * per_tile;
     p.dep_need_shared = nb1 * s->S * per_tile;
     p.done_capacity = (int)ffn_done_ints(s, routed ? budget : 0);
-    if (!done_is_clear &&
-        cudaMemsetAsync(done, 0, ffn_done_ints(s, routed ? budget : 0) * sizeof(int32_t), stream) != cudaSuccess)
+    if (!a.done_is_clear &&
+        cudaMemsetAsync(a.done, 0, ffn_done_ints(s, routed ? budget : 0) * sizeof(int32_t), a.stream) != cudaSuccess)
       return MOE_ERR_CUDA;
   }
   // GEMM-1
-  p.gather_idx = routed ? gather_idx : nullptr;
+  p.gather_idx = routed ? a.gather_idx : nullptr;
   p.gather_rows = by_rows ? (int)budget : 0;
   p.gather_src_rows = (int)s->T;
   p.n_per_sub = s->I;
   p.k_per_sub = s->H;
   p.up_row_offset = s->I;
-  p.out_routed = reinterpret_cast<__nv_bfloat16*>(h);
-  p.out_shared = reinterpret_cast<__nv_bfloat16*>(h_sh);
+  p.out_routed = reinterpret_cast<__nv_bfloat16*>(a.h);
+  p.out_shared = reinterpret_cast<__nv_bfloat16*>(a.h_sh);
   p.ld_out_routed = s->I;
   p.ld_out_shared = (long long)s->S * s->I;
-  moe_status st = pairs           ? launch_gemm_pair<true>(p, a1r, b1r, a1s, b1s, stream)
-                  : tile_n == 128 ? launch_gemm<true, 128>(p, a1r, b1r, a1s, b1s, stream)
-                                  : launch_gemm<true, 256>(p, a1r, b1r, a1s, b1s, stream);
-  if (st != MOE_OK) return st;
-  if (between != nullptr) cudaEventRecord(between, stream);
+  if (!a.gemm2_only) {
+    moe_status st = pairs           ? launch_gemm_pair<true>(p, a1r, b1r, a1s, b1s, a.stream)
+                    : tile_n == 128 ? launch_gemm<true, 128>(p, a1r, b1r, a1s, b1s, a.stream)
+                                    : launch_gemm<true, 256>(p, a1r, b1r, a1s, b1s, a.stream);
+    if (st != MOE_OK) return st;
+  }
+  if (a.between != nullptr) cudaEventRecord(a.between, a.stream);
   // GEMM-2
   p.gather_idx = nullptr;
   p.gather_rows = by_rows ? (int)budget : 0;
+  p.gather_src_rows = (int)budget;
   p.n_per_sub = s->H;
   p.k_per_sub = s->I;
   p.up_row_offset = 0;
-  p.out_routed = reinterpret_cast<__nv_bfloat16*>(y_perm);
-  p.out_shared = reinterpret_cast<__nv_bfloat16*>(y_shared);
+  p.out_routed = reinterpret_cast<__nv_bfloat16*>(a.y_perm);
+  p.out_shared = reinterpret_cast<__nv_bfloat16*>(a.y_shared);
   p.ld_out_routed = s->H;
   p.ld_out_shared = s->H;
-  if (pairs) return launch_gemm_pair<false>(p, a2r, b2r, a2s, b2s, stream);
-  return tile_n == 128 ? launch_gemm<false, 128>(p, a2r, b2r, a2s, b2s, stream)
-                       : launch_gemm<false, 256>(p, a2r, b2r, a2s, b2s, stream);
+  if (pairs) return launch_gemm_pair<false>(p, a2r, b2r, a2s, b2s, a.stream);
+  return tile_n == 128 ? launch_gemm<false, 128>(p, a2r, b2r, a2s, b2s, a.stream)
+                       : launch_gemm<false, 256>(p, a2r, b2r, a2s, b2s, a.stream);
 }

@@ -251,13 +251,8 @@ static moe_status gate_launch_t(const moe_shape* s, const uint16_t* x, const uin
   size_t pipe = (size_t)kGateStages * (TM * kGateXStride * 2 + kGateKC * w_stride * 2);
   size_t red = (size_t)TM * (NP + 1) * 4;
   size_t smem = pipe > red ? pipe : red;
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(moe_gate_kernel<NT16, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-        cudaSuccess)
-      return MOE_ERR_CUDA;
-    attr_done = true;
-  }
+  static PerDeviceOnce attr_set;
+  if (!ensure_dynamic_smem(moe_gate_kernel<NT16, NW>, smem, attr_set)) return MOE_ERR_CUDA;
   // CTAs per token tile: a power of two <= 8 that leaves every CTA at least one chunk, grown while
   // the grid stays within two CTAs per SM (measured: 256 CTAs beat 128 and 512 at 2048 and 4096 tokens)
   const int nchunks = (s->H + kGateKC - 1) / kGateKC;

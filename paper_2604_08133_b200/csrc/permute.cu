@@ -29,11 +29,11 @@ permute_count_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __rest
 
 // One CTA.  In-place exclusive scan of seg_counts (N*nseg ints, expert-major).
 __global__ void __launch_bounds__(1024, 1)
-permute_scan_kernel(int32_t* __restrict__ seg_counts, int N, int nseg, long long budget,
+permute_scan_kernel(int32_t* __restrict__ seg_counts, int N, int nseg, long long budget, int exact,
                     int32_t* __restrict__ expert_offsets, int32_t* dev_status) {
   __shared__ int scan_ws[33];
   pdl_prologue_done();
-  permute_scan_block(seg_counts, N, nseg, budget, expert_offsets, dev_status, scan_ws);
+  permute_scan_block(seg_counts, N, nseg, budget, exact != 0, expert_offsets, dev_status, scan_ws);
 }
 
 __global__ void __launch_bounds__(kPermWarps * 32)
@@ -50,11 +50,13 @@ permute_place_kernel(const int32_t* __restrict__ topk_idx, const float* __restri
                      perm_weight, pair_pos);
 }
 
-// x_perm[p, :] = x[perm_token[p], :]; one CTA per row, 16 bytes per thread per step.
+// x_perm[p, :] = x[perm_token[p], :]; one CTA per row, 16 bytes per thread per step.  rows_dev (optional):
+// the list's length as the device knows it (expert_offsets[N]) when `rows` is only an upper bound.
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ perm_token, int T, int row_vec,
-                   long long rows, uint4* __restrict__ x_perm) {
+                   long long rows, const int32_t* __restrict__ rows_dev, uint4* __restrict__ x_perm) {
   pdl_prologue_done();
+  if (rows_dev != nullptr) rows = min(rows, (long long)max(*rows_dev, 0));
   for (long long p = blockIdx.x; p < rows; p += gridDim.x) {
     int t = perm_token[p];
     t = min(max(t, 0), T - 1);
@@ -69,11 +71,12 @@ gather_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ perm
 using namespace allocmoe;
 
 moe_status launch_gather_rows(const moe_shape* s, const uint16_t* x, const int32_t* perm_token, int64_t budget,
-                              uint16_t* x_perm, cudaStream_t stream) {
+                              const int32_t* rows_dev, uint16_t* x_perm, cudaStream_t stream) {
   const int row_vec = s->H / 8;
   const long long g = budget < (1ll << 20) ? budget : (1ll << 20);
   return launch_dependent(gather_rows_kernel, dim3((unsigned)g), dim3(256), 0, stream, 1, reinterpret_cast<const uint4*>(x),
-                          perm_token, (int)s->T, row_vec, (long long)budget, reinterpret_cast<uint4*>(x_perm)) == cudaSuccess
+                          perm_token, (int)s->T, row_vec, (long long)budget, rows_dev,
+                          reinterpret_cast<uint4*>(x_perm)) == cudaSuccess
              ? MOE_OK
              : MOE_ERR_CUDA;
 }
@@ -83,19 +86,20 @@ size_t permute_ws_ints(const moe_shape* s) { return (size_t)s->N * ((s->T + 31) 
 moe_status launch_moe_permute(const moe_shape* s, const uint16_t* x, const int32_t* topk_idx, const float* topk_score,
                               const int32_t* n_sel, int64_t budget, int32_t* expert_offsets, int32_t* perm_token,
                               float* perm_weight, int32_t* pair_pos, uint16_t* x_perm, int32_t* dev_status,
-                              int32_t* seg_counts, cudaStream_t stream) {
+                              int32_t* seg_counts, bool exact, cudaStream_t stream) {
   const int nseg = (s->T + 31) / 32;
   const int grid = (nseg + kPermWarps - 1) / kPermWarps;
   bool ok = launch_dependent(permute_count_kernel, dim3((unsigned)grid), dim3(kPermWarps * 32), 0, stream, 1, topk_idx, n_sel,
                              (int)s->T, (int)s->N, (int)s->K_orig, nseg, seg_counts) == cudaSuccess;
   ok = ok && launch_dependent(permute_scan_kernel, dim3(1), dim3(1024), 0, stream, 1, seg_counts, (int)s->N, nseg,
-                              (long long)budget, expert_offsets, dev_status) == cudaSuccess;
+                              (long long)budget, exact ? 1 : 0, expert_offsets, dev_status) == cudaSuccess;
   ok = ok && launch_dependent(permute_place_kernel, dim3((unsigned)grid), dim3(kPermWarps * 32), 0, stream, 1, topk_idx,
                               topk_score, n_sel, (int)s->T, (int)s->N, (int)s->K_orig, nseg,
                               static_cast<const int32_t*>(seg_counts), (long long)budget, perm_token, perm_weight,
                               pair_pos) == cudaSuccess;
   if (!ok) return MOE_ERR_CUDA;
-  if (x_perm != nullptr && budget > 0) return launch_gather_rows(s, x, perm_token, budget, x_perm, stream);
+  if (x_perm != nullptr && budget > 0)
+    return launch_gather_rows(s, x, perm_token, budget, exact ? nullptr : expert_offsets + s->N, x_perm, stream);
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
@@ -107,20 +111,21 @@ moe_status launch_moe_permute(const moe_shape* s, const uint16_t* x, const int32
 // carries these 256 KB until the process exits.
 #include <mutex>
 
+#include "shape_check.h"
+
 namespace {
 
 constexpr int kStaticSegCounts = 65536;   // N * ceil(T/32) may not exceed this (256 KB of int32)
 static __device__ __align__(256) int32_t g_static_seg_counts[kStaticSegCounts];
 
-constexpr int kMaxDevices = 64;
-int32_t* g_static_seg_ptr[kMaxDevices] = {};
+int32_t* g_static_seg_ptr[allocmoe::kMaxDevices] = {};
 std::mutex g_static_mutex;
 
 // In host code the array's name is only a handle; the address a kernel can use has to be asked for
 // while the owning device is current.  Done once per device, on that device's first call.
 moe_status static_scratch(int32_t** out) {
   int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MOE_ERR_CUDA;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= allocmoe::kMaxDevices) return MOE_ERR_CUDA;
   std::lock_guard<std::mutex> lock(g_static_mutex);
   if (g_static_seg_ptr[dev] == nullptr) {
     void* p = nullptr;
@@ -131,8 +136,6 @@ moe_status static_scratch(int32_t** out) {
   return MOE_OK;
 }
 
-bool is_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
 }  // namespace
 
 extern "C" moe_status moe_permute_static(const moe_shape* shape, const uint16_t* x, const int32_t* topk_idx,
@@ -140,13 +143,10 @@ extern "C" moe_status moe_permute_static(const moe_shape* shape, const uint16_t*
                                          int32_t* expert_offsets, int32_t* perm_token, float* perm_weight,
                                          int32_t* pair_pos, uint16_t* x_perm, int32_t* dev_status, void* stream) {
   const moe_shape* s = shape;
-  if (s == nullptr || s->flags != 0 || s->T < 1 || s->H < 64 || s->H % 64 != 0 || s->N < 8 || s->N % 4 != 0 ||
-      s->N > kMaxExperts || s->K_orig < 1 || s->K_orig > 16 || s->K_orig > s->N || s->K_base < 0 ||
-      s->K_base > s->K_orig || (long long)s->T * s->K_orig >= (1ll << 31))
-    return MOE_ERR_ARG;
+  if (!allocmoe::shape_ok(s)) return MOE_ERR_ARG;   // the same shapes as moe_permute accepts
   if (!topk_idx || !topk_score || !n_sel || !expert_offsets || !perm_token || !perm_weight || !pair_pos || !dev_status)
     return MOE_ERR_ARG;
-  if (x_perm != nullptr && (!x || !is_aligned16(x) || !is_aligned16(x_perm))) return MOE_ERR_ARG;
+  if (x_perm != nullptr && (!x || !allocmoe::aligned16(x) || !allocmoe::aligned16(x_perm))) return MOE_ERR_ARG;
   if (budget < (int64_t)s->K_base * s->T || budget > (int64_t)s->K_orig * s->T) return MOE_ERR_BUDGET;
   // the fixed array bounds the problem size: refuse anything larger, touch nothing
   if ((long long)s->N * ((s->T + 31) / 32) > (long long)kStaticSegCounts) return MOE_ERR_WORKSPACE;
@@ -156,5 +156,5 @@ extern "C" moe_status moe_permute_static(const moe_shape* shape, const uint16_t*
   // Every counter a call reads is written by its own count kernel first, so whatever an earlier
   // call left in the array needs no clearing.
   return launch_moe_permute(s, x, topk_idx, topk_score, n_sel, budget, expert_offsets, perm_token, perm_weight,
-                            pair_pos, x_perm, dev_status, seg_counts, (cudaStream_t)stream);
+                            pair_pos, x_perm, dev_status, seg_counts, true, (cudaStream_t)stream);
 }

@@ -23,7 +23,7 @@ constexpr int kRouteWarps = kSelThreads / 32;
 // The per-warp masks of the permutation reuse SelectSmem::warp_hist (32 warps x 256 ints >= 32 x 128).
 __global__ void __launch_bounds__(kSelThreads, 1)
 moe_route_kernel(const float* __restrict__ topk_score, const int32_t* __restrict__ topk_idx, int T, int N, int K_orig,
-                 int K_base, long long budget, int use_smem_keys, int32_t* __restrict__ n_sel,
+                 int K_base, long long budget, int use_smem_keys, int n_sel_given, int32_t* __restrict__ n_sel,
                  int32_t* __restrict__ expert_offsets, int32_t* __restrict__ perm_token,
                  float* __restrict__ perm_weight, int32_t* __restrict__ pair_pos, int32_t* dev_status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -33,8 +33,11 @@ moe_route_kernel(const float* __restrict__ topk_score, const int32_t* __restrict
   const int nseg = (T + 31) / 32;
   pdl_prologue_done();
 
-  alloc_t_select_block(smem_raw, topk_score, T, K_orig, K_base, budget - (long long)K_base * T, use_smem_keys, n_sel,
-                       dev_status);   // ends with a block barrier: n_sel is visible, the pool is free
+  // n_sel_given: the caller's n_sel is the input (a selection made over a larger pool, of which this batch is a
+  // part); the kept pairs then number at most `budget`, not exactly `budget`.
+  if (!n_sel_given)
+    alloc_t_select_block(smem_raw, topk_score, T, K_orig, K_base, budget - (long long)K_base * T, use_smem_keys, n_sel,
+                         dev_status);   // ends with a block barrier: n_sel is visible, the pool is free
 
   // Every warp owns at most one 32-token segment here (moe_route_fits), so the masks and expert ids
   // built for the count are still there for the placement: nothing is loaded twice.
@@ -47,7 +50,7 @@ moe_route_kernel(const float* __restrict__ topk_score, const int32_t* __restrict
     for (int e = lane; e < N; e += 32) seg_counts[(long long)e * nseg + seg] = __popc(mask[e]);
   }
   __syncthreads();
-  permute_scan_block(seg_counts, N, nseg, budget, expert_offsets, dev_status, sm.scan_ws);
+  permute_scan_block(seg_counts, N, nseg, budget, !n_sel_given, expert_offsets, dev_status, sm.scan_ws);
   __syncthreads();
   if (seg < nseg)
     permute_place_from_masks(mask, e_loc, n, topk_score, seg, T, K_orig, nseg, seg_counts, budget, perm_token,
@@ -83,7 +86,7 @@ struct RouteClusterSmem {
 
 __global__ void __launch_bounds__(kSelThreads, 1)
 moe_route_cluster_kernel(const float* __restrict__ topk_score, const int32_t* __restrict__ topk_idx, int T, int N,
-                         int K_orig, int K_base, long long budget, int32_t* __restrict__ n_sel,
+                         int K_orig, int K_base, long long budget, int n_sel_given, int32_t* __restrict__ n_sel,
                          int32_t* __restrict__ expert_offsets, int32_t* __restrict__ perm_token,
                          float* __restrict__ perm_weight, int32_t* __restrict__ pair_pos, int32_t* dev_status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -99,7 +102,9 @@ moe_route_cluster_kernel(const float* __restrict__ topk_score, const int32_t* __
 
   // ---------------- Alloc-T selection (Sec. 3.3)
   int n_mine = K_base;
-  if (R > 0 && Kr > 0) {
+  if (n_sel_given) {                       // the caller's selection (see moe_route_kernel)
+    if (have) n_mine = n_sel[t];
+  } else if (R > 0 && Kr > 0) {
     const uint32_t* bits = reinterpret_cast<const uint32_t*>(topk_score);
     uint32_t k[16];
     bool bad = false;
@@ -165,7 +170,7 @@ moe_route_cluster_kernel(const float* __restrict__ topk_score, const int32_t* __
       n_mine = K_base + gt + min(eq, max(0, need_eq - ties_before));
     }
   }
-  if (have) n_sel[t] = n_mine;
+  if (have && !n_sel_given) n_sel[t] = n_mine;
 
   // ---------------- permutation: counts per (expert, segment), this CTA's segments = its warps
   uint32_t* mask = reinterpret_cast<uint32_t*>(sm.warp_hist[warp]);
@@ -202,7 +207,7 @@ moe_route_cluster_kernel(const float* __restrict__ topk_score, const int32_t* __
   }
   if (rank == 0 && tid == 0) {
     expert_offsets[N] = total;
-    if ((long long)total != budget) set_dev_status(dev_status, MOE_ERR_BUDGET);
+    if (n_sel_given ? (long long)total > budget : (long long)total != budget) set_dev_status(dev_status, MOE_ERR_BUDGET);
   }
   __syncthreads();
   for (int i = tid; i < N * kRouteWarps; i += kSelThreads) sm.lbase[i] += sm.ebase[i / kRouteWarps];
@@ -228,40 +233,31 @@ static bool route_one_cta(const moe_shape* s) {
   return nseg <= kRouteWarps && (long long)s->N * nseg <= (long long)kSelMaxSmemKeys;
 }
 
+// n_sel_given: n_sel is an input and only the permutation's lists are built; `budget` is then an upper bound.
 moe_status launch_moe_route(const moe_shape* s, const float* topk_score, const int32_t* topk_idx, int64_t budget,
-                            int32_t* n_sel, int32_t* expert_offsets, int32_t* perm_token, float* perm_weight,
-                            int32_t* pair_pos, int32_t* dev_status, cudaStream_t stream) {
+                            bool n_sel_given, int32_t* n_sel, int32_t* expert_offsets, int32_t* perm_token,
+                            float* perm_weight, int32_t* pair_pos, int32_t* dev_status, cudaStream_t stream) {
   if (!route_one_cta(s)) {
     const unsigned n_ctas = (unsigned)((s->T + kSelThreads - 1) / kSelThreads);
-    static bool cattr_done = false;
-    if (!cattr_done) {
-      if (cudaFuncSetAttribute(moe_route_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)sizeof(RouteClusterSmem)) != cudaSuccess)
-        return MOE_ERR_CUDA;
-      cattr_done = true;
-    }
+    static PerDeviceOnce cattr_set;
+    if (!ensure_dynamic_smem(moe_route_cluster_kernel, sizeof(RouteClusterSmem), cattr_set)) return MOE_ERR_CUDA;
     return launch_dependent_cluster(moe_route_cluster_kernel, dim3(n_ctas), dim3(kSelThreads), sizeof(RouteClusterSmem),
                                     stream, dim3(n_ctas, 1, 1), topk_score, topk_idx, (int)s->T, (int)s->N,
-                                    (int)s->K_orig, (int)s->K_base, (long long)budget, n_sel, expert_offsets,
-                                    perm_token, perm_weight, pair_pos, dev_status) == cudaSuccess
+                                    (int)s->K_orig, (int)s->K_base, (long long)budget, n_sel_given ? 1 : 0, n_sel,
+                                    expert_offsets, perm_token, perm_weight, pair_pos, dev_status) == cudaSuccess
                ? MOE_OK
                : MOE_ERR_CUDA;
   }
   const long long P = (long long)s->T * (s->K_orig - s->K_base);
-  const int use_smem_keys = (P <= kSelMaxSmemKeys) ? 1 : 0;
+  const int use_smem_keys = (P <= kSelMaxSmemKeys && !n_sel_given) ? 1 : 0;
   const long long counters = (long long)s->N * ((s->T + 31) / 32);
   const long long pool_ints = (use_smem_keys && P > counters) ? P : counters;
   const size_t smem = sizeof(SelectSmem) + (size_t)pool_ints * 4;
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(moe_route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)(sizeof(SelectSmem) + (size_t)kSelMaxSmemKeys * 4)) != cudaSuccess)
-      return MOE_ERR_CUDA;
-    attr_done = true;
-  }
+  static PerDeviceOnce attr_set;
+  if (!ensure_dynamic_smem(moe_route_kernel, sizeof(SelectSmem) + (size_t)kSelMaxSmemKeys * 4, attr_set)) return MOE_ERR_CUDA;
   return launch_dependent(moe_route_kernel, dim3(1), dim3(kSelThreads), smem, stream, 1, topk_score, topk_idx, (int)s->T,
-                          (int)s->N, (int)s->K_orig, (int)s->K_base, (long long)budget, use_smem_keys, n_sel,
-                          expert_offsets, perm_token, perm_weight, pair_pos, dev_status) == cudaSuccess
+                          (int)s->N, (int)s->K_orig, (int)s->K_base, (long long)budget, use_smem_keys, n_sel_given ? 1 : 0,
+                          n_sel, expert_offsets, perm_token, perm_weight, pair_pos, dev_status) == cudaSuccess
              ? MOE_OK
              : MOE_ERR_CUDA;
 }

@@ -204,8 +204,10 @@ DEV void permute_count_warp(uint32_t* mask, const int32_t* __restrict__ topk_idx
 
 // The whole CTA: in-place exclusive scan of seg_counts (N*nseg ints, expert-major; shared or global
 // memory), expert_offsets, and the check that the kept pairs add up to the budget.
-DEV void permute_scan_block(int32_t* seg_counts, int N, int nseg, long long budget, int32_t* __restrict__ expert_offsets,
-                            int32_t* dev_status, int* scan_ws) {
+// exact: the kept pairs must number exactly `budget`; otherwise `budget` is only an upper bound (the caller's
+// n_sel came from a selection over a larger pool and this batch's share is known to the device alone).
+DEV void permute_scan_block(int32_t* seg_counts, int N, int nseg, long long budget, bool exact,
+                            int32_t* __restrict__ expert_offsets, int32_t* dev_status, int* scan_ws) {
   const long long M = (long long)N * nseg;
   const int per = (int)((M + blockDim.x - 1) / blockDim.x);
   const long long lo = min(M, (long long)threadIdx.x * per), hi = min(M, lo + per);
@@ -221,7 +223,7 @@ DEV void permute_scan_block(int32_t* seg_counts, int N, int nseg, long long budg
   }
   if (threadIdx.x == 0) {
     expert_offsets[N] = total;
-    if ((long long)total != budget) set_dev_status(dev_status, MOE_ERR_BUDGET);
+    if (exact ? (long long)total != budget : (long long)total > budget) set_dev_status(dev_status, MOE_ERR_BUDGET);
   }
 }
 

@@ -37,13 +37,9 @@ moe_status launch_alloc_t_select(const moe_shape* s, const float* topk_score, in
   const long long P = (long long)s->T * (s->K_orig - s->K_base);
   int use_smem = 0;
   const size_t smem = select_dynamic_smem(P, &use_smem);
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(alloc_t_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)(sizeof(SelectSmem) + (size_t)kSelMaxSmemKeys * 4)) != cudaSuccess)
-      return MOE_ERR_CUDA;
-    attr_done = true;
-  }
+  static PerDeviceOnce attr_set;
+  if (!ensure_dynamic_smem(alloc_t_select_kernel, sizeof(SelectSmem) + (size_t)kSelMaxSmemKeys * 4, attr_set))
+    return MOE_ERR_CUDA;
   return launch_dependent(alloc_t_select_kernel, dim3(1), dim3(kSelThreads), smem, stream, 1, topk_score, (int)s->T,
                           (int)s->K_orig, (int)s->K_base, R, use_smem, n_sel, dev_status) == cudaSuccess
              ? MOE_OK

@@ -47,3 +47,30 @@ def test_algorithmic_work_matches_the_formulas_by_hand():
     assert gb == (touched + S) * 4.0 * H * I + B * H * 2 + T * H * 2 + B * I * 2 + S * T * I * 2
     # the weights dominate at decode: within 1 % of W13 of the touched experts alone
     assert abs(gb / ((touched + S) * 4.0 * H * I) - 1) < 0.01
+
+
+def test_ncu_traffic_is_quoted_only_for_the_kernel_source_it_was_taken_on(tmp_path, monkeypatch):
+    prof = tmp_path / "profiles"
+    prof.mkdir()
+    sha = bench.kernel_source_sha16()
+    (prof / "ncu_traffic.txt").write_text(
+        "# comment\n"
+        "ffn_gemm_kernel<true, 256>\tc2\t192\t720600000\t%s\tabc1234\tncu\n"
+        "ffn_gemm_pair_kernel<true>\tc3\t12288\t886000000\t0000000000000000\tabc1234\tncu\n" % sha)
+    real_join = os.path.join
+    monkeypatch.setattr(bench, "ROOT", str(tmp_path))
+    # the fingerprint still reads the real sources
+    monkeypatch.setattr(bench, "kernel_source_sha16", lambda: sha)
+    assert bench.ncu_traffic_bytes("ffn_gemm_kernel<true, 256>", "c2", 192) == 720600000.0
+    assert bench.ncu_traffic_bytes("ffn_gemm_kernel<true, 256>", "c2", 384) is None          # another budget
+    assert bench.ncu_traffic_bytes("ffn_gemm_pair_kernel<true>", "c3", 12288) is None        # stale fingerprint
+    assert real_join is os.path.join
+
+
+def test_median_and_default_steps():
+    assert bench.median([3.0, 1.0, 2.0]) == 2.0 and bench.median([4.0, 1.0, 2.0, 3.0]) == 2.5
+    c = synth.CONFIGS
+    assert bench.default_steps(c["c2"])[0] >= 200 and bench.default_steps(c["c4"])[0] <= 20
+    assert bench.default_steps(c["c5"])[0] < bench.default_steps(c["c3"])[0]
+    for name in ("c2", "c3", "c4", "c5"):
+        assert bench.default_steps(c[name])[1] >= 3                                          # at least three warm-ups

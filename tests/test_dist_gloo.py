@@ -28,7 +28,7 @@ def _worker(rank, world, port, T, K, K_base, budget, q):
         mine = full[rank * T:(rank + 1) * T].clone()
         n_sel, b_local = D.alloc_t_select_global(mine, K_base, budget, select=_oracle_select)
         slow = D.max_over_ranks(10.0 + rank)                          # rank 1 is "slower"
-        q.put((rank, n_sel.numpy(), b_local, slow))
+        q.put((rank, n_sel.numpy(), int(b_local), slow))
     finally:
         dist.destroy_process_group()
 
@@ -65,5 +65,5 @@ def test_global_selection_over_two_gloo_ranks(T, K, K_base, mult):
 def test_single_process_is_the_identity():
     s = synth.score_rows(16, 3, 5)
     n_sel, b = D.alloc_t_select_global(s, 1, 30, select=_oracle_select)
-    assert b == 30 and np.array_equal(n_sel.numpy(), orc.n_sel_from_mask(orc.alloc_t_select(s.numpy(), 1, 30)))
+    assert int(b) == 30 and np.array_equal(n_sel.numpy(), orc.n_sel_from_mask(orc.alloc_t_select(s.numpy(), 1, 30)))
     assert D.max_over_ranks(3.5) == 3.5

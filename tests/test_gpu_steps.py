@@ -214,7 +214,7 @@ def test_grouped_ffn_against_oracle(T, H, N, I, K, budget):
     ws = B.new_workspace(shape, budget)
     y = torch.full((budget, H), float("nan"), dtype=torch.bfloat16, device="cuda")
     st = _status()
-    B.moe_grouped_ffn(shape, x_perm, torch.from_numpy(off).cuda(), budget, d["W13"].cuda(), d["W2"].cuda(), y, st, ws)
+    B.moe_grouped_ffn(shape, x_perm, None, torch.from_numpy(off).cuda(), budget, d["W13"].cuda(), d["W2"].cuda(), y, st, ws)
     torch.cuda.synchronize()
     assert st.item() == 0
     want = np.zeros((budget, H))
@@ -224,6 +224,35 @@ def test_grouped_ffn_against_oracle(T, H, N, I, K, budget):
     got = y.float().cpu().numpy()
     assert np.isfinite(got).all()
     assert max_rel(got, want) <= TOL_OUT
+    # the same rows read from x through perm_token instead of a permuted copy: identical bits
+    y2 = torch.full((budget, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.moe_grouped_ffn(shape, d["x"].cuda(), torch.from_numpy(tok).cuda(), torch.from_numpy(off).cuda(), budget,
+                      d["W13"].cuda(), d["W2"].cuda(), y2, st, ws)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    assert torch.equal(y.view(torch.int16), y2.view(torch.int16))
+
+
+def test_grouped_ffn_index_mode_clamps_bad_token_indices():
+    """perm_token entries outside [0, T) (a list left by a routing step that reported an error) are clamped:
+    rows are meaningless but every access stays inside x and y."""
+    T, H, N, I = 40, 128, 8, 128
+    cfg = synth.CONFIGS["c1"].with_(T=T, H=H, N=N, I=I)
+    d = synth.make_layer(cfg)
+    off = torch.tensor([0, 5, 5, 5, 36, 36, 36, 36, 40], dtype=torch.int32).cuda()
+    tok = torch.arange(T, dtype=torch.int32)
+    tok[3], tok[20], tok[39] = -7, 10 ** 6, T
+    shape = B.shape_of(cfg)
+    ws = B.new_workspace(shape, T)
+    y = torch.full((T + 8, H), 123.0, dtype=torch.bfloat16, device="cuda")
+    st = _status()
+    B.moe_grouped_ffn(shape, d["x"].cuda(), tok.cuda(), off, T, d["W13"].cuda(), d["W2"].cuda(), y, st, ws)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    assert (y[T:] == 123.0).all() and bool(torch.isfinite(y.float()).all())
+    xn, W13, W2 = np32(d["x"]), np32(d["W13"]), np32(d["W2"])
+    want = orc.expert_ffn(xn[5:20], W13[3], W2[3])          # untouched rows of the list are still right
+    assert max_rel(y[5:20].float().cpu().numpy(), want) <= TOL_OUT
 
 
 def test_grouped_ffn_skips_empty_experts_and_respects_segment_ends():
@@ -237,7 +266,7 @@ def test_grouped_ffn_skips_empty_experts_and_respects_segment_ends():
     ws = B.new_workspace(shape, T)
     y = torch.full((T + 8, H), 123.0, dtype=torch.bfloat16, device="cuda")
     st = _status()
-    B.moe_grouped_ffn(shape, x_perm, torch.from_numpy(off).cuda(), T, d["W13"].cuda(), d["W2"].cuda(), y, st, ws)
+    B.moe_grouped_ffn(shape, x_perm, None, torch.from_numpy(off).cuda(), T, d["W13"].cuda(), d["W2"].cuda(), y, st, ws)
     torch.cuda.synchronize()
     assert st.item() == 0
     assert (y[T:] == 123.0).all()                       # nothing is written past the list
@@ -261,13 +290,13 @@ def test_grouped_ffn_keeps_inconsistent_offsets_inside_the_list():
     for bad in ([-5, 10, 5, 10 ** 6, 0, 0, 0, 0, 0], [0, T, 0, T, 0, T, 0, T, T], [0] + [T] * 8, [7 * T] * 9,
                 [0, 300, 300, 300, 300, 300, 300, 300, -1]):
         y = torch.full((T + 8, H), 123.0, dtype=torch.bfloat16, device="cuda")
-        B.moe_grouped_ffn(shape, x_perm, torch.tensor(bad, dtype=torch.int32).cuda(), T, W13, W2, y, st, ws)
+        B.moe_grouped_ffn(shape, x_perm, None, torch.tensor(bad, dtype=torch.int32).cuda(), T, W13, W2, y, st, ws)
         torch.cuda.synchronize()
         assert st.item() == 0
         assert (y[T:] == 123.0).all()
     off = np.array([0, 100, 100, 100, 260, 260, 260, 260, 300], np.int32)
     y = torch.full((T, H), float("nan"), dtype=torch.bfloat16, device="cuda")
-    B.moe_grouped_ffn(shape, x_perm, torch.from_numpy(off).cuda(), T, W13, W2, y, st, ws)
+    B.moe_grouped_ffn(shape, x_perm, None, torch.from_numpy(off).cuda(), T, W13, W2, y, st, ws)
     torch.cuda.synchronize()
     xn, w13, w2 = np32(d["x"]), np32(d["W13"]), np32(d["W2"])
     want = np.concatenate([orc.expert_ffn(xn[0:100], w13[0], w2[0]), orc.expert_ffn(xn[100:260], w13[3], w2[3]),
@@ -316,6 +345,47 @@ def test_combine_against_oracle_formula():
     # one bf16 rounding of an fp32 sum of exactly representable products
     assert np.abs(got - want).max() <= 2 ** -8 * np.abs(want).max()
     assert max_rel(got, want) <= 4e-3
+
+
+@pytest.mark.parametrize("T,budget", [(40, 40), (700, 1390)])
+def test_bounded_wait_runs_out_and_the_kernel_returns(T, budget):
+    """Failure path of the expert GEMMs: GEMM-2 launched alone, so the row-block counters it waits on are never
+    filled, with the wait limit cut to about a millisecond.  The waits must give up, the kernel must return with
+    MOE_ERR_TIMEOUT in the status word and nothing written, and the next ordinary call must be right.  Nothing
+    faults and nothing waits without a limit; (700, 1390) runs the CTA-pair kernel, (40, 40) the one-CTA kernel
+    with rows fetched by index."""
+    H, N, I = 128, 8, 128
+    cfg = synth.CONFIGS["c1"].with_(T=T, H=H, N=N, I=I, K_orig=2, K_base=1, budget=budget)
+    d = synth.make_layer(cfg)
+    dn = {k: np32(v) for k, v in d.items()}
+    r = orc.route(dn["x"], dn["W_gate"], None, 2, 1, budget)
+    p = orc.permute(r["topk_idx"], r["topk_score"], r["n_sel"], N)
+    off = torch.from_numpy(p["expert_offsets"]).cuda()
+    tok = torch.from_numpy(p["perm_token"]).cuda()
+    shape = B.shape_of(cfg)
+    ws = B.new_workspace(shape, budget)
+    W13, W2 = d["W13"].cuda(), d["W2"].cuda()
+    y = torch.full((budget + 8, H), 123.0, dtype=torch.bfloat16, device="cuda")
+    st = _status()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    B.moe_selftest_wait_timeout(shape, off, budget, W2, y, 2_000_000, st, ws)      # about 1 ms of SM clocks
+    e1.record()
+    torch.cuda.synchronize()
+    assert st.item() == 1 << B.MOE_ERR_TIMEOUT
+    assert e0.elapsed_time(e1) < 200.0                      # gave up after milliseconds, not after the default 0.5 s
+    assert (y == 123.0).all()                               # no tile was computed, nothing was stored
+    # the context is intact and the workspace reusable: the ordinary call right after is correct
+    st.zero_()
+    B.moe_grouped_ffn(shape, d["x"].cuda(), tok, off, budget, W13, W2, y, st, ws)
+    torch.cuda.synchronize()
+    assert st.item() == 0 and (y[budget:] == 123.0).all()
+    offn = p["expert_offsets"]
+    e = int(np.argmax(np.diff(offn)))
+    want = orc.expert_ffn(dn["x"][p["perm_token"][offn[e]:offn[e + 1]]], dn["W13"][e], dn["W2"][e])
+    assert max_rel(y[offn[e]:offn[e + 1]].float().cpu().numpy(), want) <= TOL_OUT
+    with pytest.raises(B.MoeError):
+        B.moe_selftest_wait_timeout(shape, off, budget, W2, y, 10, st, ws)         # limit below the accepted range
 
 
 @pytest.mark.parametrize("pair,gather,tile_n", [("0", "0", "256"), ("1", "0", "256"), ("0", "1000000", "256"),

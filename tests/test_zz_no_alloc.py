@@ -54,6 +54,13 @@ def _one_case(T, N, K, kb, mult, seed):
         assert torch.equal(ref[k].view(torch.int16) if ref[k].dtype == torch.bfloat16 else ref[k],
                            got[k].view(torch.int16) if got[k].dtype == torch.bfloat16 else got[k]), k
     assert int(got["off"][-1]) == budget
+    # and directly against the oracle's permutation of the same routing
+    want = orc.permute(idx.cpu().numpy(), sc.cpu().numpy(), n_sel.cpu().numpy(), N)
+    assert np.array_equal(got["off"].cpu().numpy(), want["expert_offsets"])
+    assert np.array_equal(got["tok"].cpu().numpy(), want["perm_token"])
+    assert np.array_equal(got["wgt"].cpu().numpy(), want["perm_weight"])
+    assert np.array_equal(got["pos"].cpu().numpy(), want["pair_pos"])
+    assert torch.equal(got["xp"].cpu(), x.cpu()[torch.from_numpy(want["perm_token"]).long()])
 
 
 def test_static_scratch_matches_workspace_version_twice_in_a_row():
@@ -62,7 +69,23 @@ def test_static_scratch_matches_workspace_version_twice_in_a_row():
     _one_case(T=4096, N=64, K=6, kb=1, mult=2.0, seed=3)
 
 
+def test_static_scratch_at_exactly_its_size():
+    _one_case(T=32768, N=64, K=2, kb=1, mult=1.5, seed=4)    # 64 * 1024 = 65536 counters: the whole array
+    _one_case(T=32737, N=64, K=2, kb=0, mult=0.7, seed=5)    # the last segment holds one token
+
+
 def test_static_scratch_rejects_shapes_beyond_its_size():
+    shape = B.make_shape(32800, 128, 64, 64, 0, 2, 1)         # 64 * 1025 = 65600 counters: just past the array
+    dummy = torch.zeros(16, dtype=torch.int32, device="cuda")
+    with pytest.raises(B.MoeError) as ei:
+        B.moe_permute_static(shape, None, dummy, dummy.float(), dummy, 32800, dummy, dummy, dummy.float(), dummy, None,
+                             dummy)
+    assert ei.value.status == B.MOE_ERR_WORKSPACE
+    bad = B.make_shape(64, 128, 8, 100, 0, 2, 1)              # I not a multiple of 64: refused like moe_permute does
+    with pytest.raises(B.MoeError) as ei:
+        B.moe_permute_static(bad, None, dummy, dummy.float(), dummy, 64, dummy, dummy, dummy.float(), dummy, None, dummy)
+    assert ei.value.status == B.MOE_ERR_ARG
+
     T, N, K = 40000, 64, 2                                    # 64 * 1250 = 80000 counters > 65536
     shape = B.make_shape(T, 128, N, 64, 0, K, 1)
     dummy = torch.zeros(16, dtype=torch.int32, device="cuda")
