@@ -16,6 +16,9 @@ Passages followed
                      (K_l-K_base)*T                               -> alloc_t_select, alloc_t_select_threshold
   Sec. 3.3, last paragraph: K_base = K_l is plain Top-K routing   -> covered by tests
   Eq. 3-6 (Sec. 3.2) Alloc-L grouped-knapsack DP                  -> alloc_l_dp, alloc_l_bruteforce
+  Sec. 2 / App. A.1  the token-level rules Alloc-T is compared with: Top-P count
+                     (Dynamic-MoE) and skipping relative to the top-1 score (NAEE
+                     extended to Top-K)                            -> top_p_count, rel_threshold_count
 
 Readings where the paper is silent or inconsistent (each is listed in the design notes):
   * the candidate set holds each token's Top-K_orig pairs (the procedure paragraph's
@@ -160,6 +163,45 @@ def alloc_t_bruteforce(topk_score, K_base: int, budget: int):
     best = float(obj.max())
     arg = [allz[b].reshape(T, K).copy() for b in np.flatnonzero(np.abs(obj - best) <= 1e-15)]
     return best, arg
+
+
+# ----------------------------------------------------------------------------- token-level comparison rules
+def top_p_count(topk_score, P: float) -> np.ndarray:
+    """Top-P routing (Sec. 2; the Dynamic-MoE setting of App. A.1): a token activates experts in
+    descending score order until their cumulative score reaches P.  n_t = the smallest n >= 1 with
+    s[t,0] + ... + s[t,n-1] >= P, K_orig if the row never gets there.  The running sum and the
+    comparison are fp32, columns in order: the decision is an integer, so it is taken in the
+    precision the kernel uses."""
+    s = np.asarray(topk_score, np.float32)
+    T, K = s.shape
+    thr = np.float32(P)
+    n = np.full(T, K, np.int32)
+    for t in range(T):
+        cum = np.float32(0.0)
+        for j in range(K):
+            cum = np.float32(cum + s[t, j])
+            if cum >= thr:
+                n[t] = j + 1
+                break
+    return n
+
+
+def rel_threshold_count(topk_score, beta: float) -> np.ndarray:
+    """Expert skipping relative to the top-1 score (App. A.1, the NAEE setting extended from Top-2
+    to Top-K): the k-th expert of a token is skipped when its score is below beta times the token's
+    top-1 score.  Rows are sorted descending, so the kept experts are a prefix; the top-1 expert is
+    never skipped.  fp32 product and comparison."""
+    s = np.asarray(topk_score, np.float32)
+    T, K = s.shape
+    n = np.ones(T, np.int32)
+    for t in range(T):
+        cut = np.float32(np.float32(beta) * s[t, 0])
+        for j in range(1, K):
+            if s[t, j] >= cut:
+                n[t] = j + 1
+            else:
+                break
+    return n
 
 
 # ----------------------------------------------------------------------------- permutation
