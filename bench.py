@@ -550,10 +550,38 @@ def bench_workload(env, args, name, budget_mult, steps_arg, warmup_arg, full=Tru
                               "overlap the neighbouring steps' compute; weights resident"}
         assert int(status.item()) == 0
 
+    if full and not args.no_extras and n_layers == 1:
+        res["select_kernels_us"] = bench_select_rules(env, cfg, shape, inter["topk_score"], budget, steps)
+
     if (args.global_alloc_t or env.world > 1) and n_layers == 1 and name == args.workload:
         res["global_alloc_t"] = bench_global_alloc_t(env, cfg, shape, layers[0], budget, steps, warmup)
     res["_cfg"], res["_budget"] = cfg, budgets[0]
     return res
+
+
+def bench_select_rules(env, cfg, shape, topk_score, budget, steps):
+    """Alloc-T's selection kernel next to the two token-level rules the paper compares it with (Top-P count, skipping
+    relative to the top-1 score; thresholds calibrated off line to the same budget), on this workload's own scores:
+    device time per call in microseconds.  Speed only; the paper's accuracy comparison is out of scope."""
+    import torch
+    from paper_2604_08133_b200 import binding as B
+    from paper_2604_08133_b200 import token_baselines as TB
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    n_sel = torch.empty(cfg.T, dtype=torch.int32, device="cuda")
+    r = {}
+    fn = lambda: B.alloc_t_select(shape, topk_score, budget, n_sel, st, None)
+    fn()
+    r["alloc_t_select"] = median(env.time_blocks(fn, steps)) * 1e3
+    for rule, inc, hi in (("top_p", True, 2.0), ("rel", False, 1.5)):
+        thr, tot = TB.calibrate(TB.library_selector(rule, shape, st), topk_score, budget, increasing=inc, lo=0.0, hi=hi)
+        f = B.moe_select_top_p if rule == "top_p" else B.moe_select_rel_threshold
+        fn = lambda: f(shape, topk_score, thr, n_sel, None, st)
+        fn()
+        key = "top_p_count" if rule == "top_p" else "rel_threshold"
+        r[key] = median(env.time_blocks(fn, steps)) * 1e3
+        r[key + "_threshold"], r[key + "_kept"] = thr, tot
+    assert int(st.item()) == 0
+    return r
 
 
 def bench_global_alloc_t(env, cfg, shape, d, budget, steps, warmup):

@@ -202,6 +202,24 @@ moe_status moe_layer_forward_routed(const moe_shape* shape, const uint16_t* x, c
                                     uint16_t* out, int32_t* dev_status, void* ws, size_t ws_bytes,
                                     void* stream);
 
+/* The two token-level rules the paper measures Alloc-T against (Sec. 2, related work; App. A.1, baseline
+ * settings), with Alloc-T's output format so that moe_layer_forward_routed can run the layer on them.  They
+ * decide token by token from a threshold that those methods calibrate off line to meet a target budget;
+ * nothing is pooled, so the kept total is whatever the threshold gives (read it from `total`).
+ *   moe_select_top_p          Top-P routing: n_sel[t] = the smallest n >= 1 with
+ *                             topk_score[t,0] + ... + topk_score[t,n-1] >= P (fp32, summed in column order),
+ *                             K_orig if the row never reaches P
+ *   moe_select_rel_threshold  expert skipping relative to the top-1 score: column j >= 1 is dropped when
+ *                             topk_score[t,j] < beta * topk_score[t,0] (fp32 product); n_sel[t] counts the
+ *                             leading columns that stay, at least 1
+ *   topk_score device fp32 [T,K_orig], rows descending;  n_sel device int32 [T]
+ *   total      device int32 [1] or NULL: sum of n_sel is ADDED to it (the caller zeroes it)
+ *   dev_status MOE_ERR_NONFINITE is raised for a NaN, Inf or negative score, as in alloc_t_select */
+moe_status moe_select_top_p(const moe_shape* shape, const float* topk_score, float P, int32_t* n_sel,
+                            int32_t* total, int32_t* dev_status, void* stream);
+moe_status moe_select_rel_threshold(const moe_shape* shape, const float* topk_score, float beta, int32_t* n_sel,
+                                    int32_t* total, int32_t* dev_status, void* stream);
+
 /* Pre-norm of a residual layer stack (not part of the paper's method; the layer stack workload
  * needs it, see the stack recurrence x_{l+1} = x_l + MoE(norm(x_l))): out[t] = x[t] / sqrt(mean_h
  * x[t,h]^2 + 1e-6), unit gain, fp32 math, one bf16 rounding.  x, out device bf16 [T,H]. */

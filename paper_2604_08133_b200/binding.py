@@ -10,14 +10,15 @@ from typing import Dict, Optional
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "liballocmoe.so")
+# ALLOCMOE_LIB selects another build of the same library (the checked build, see build.py)
+LIB_PATH = os.environ.get("ALLOCMOE_LIB") or os.path.join(_PKG, "liballocmoe.so")
 
 MOE_OK, MOE_ERR_ARG, MOE_ERR_BUDGET, MOE_ERR_WORKSPACE, MOE_ERR_CUDA, MOE_ERR_NONFINITE, MOE_ERR_TIMEOUT = range(7)
 
 EXPORTS = ("moe_status_string", "moe_workspace_bytes", "moe_gate", "alloc_t_select", "moe_permute",
            "moe_grouped_ffn", "moe_shared_ffn", "moe_combine", "moe_layer_forward", "moe_layer_intermediates",
            "moe_rmsnorm", "moe_profile_enable", "moe_profile_read", "moe_permute_static", "moe_route", "alloc_l_solve",
-           "moe_layer_forward_routed", "moe_selftest_wait_timeout")
+           "moe_layer_forward_routed", "moe_selftest_wait_timeout", "moe_select_top_p", "moe_select_rel_threshold")
 PROFILE_STAGES = ("gate", "route", "gather", "ffn_gemm1", "ffn_gemm2", "combine")
 
 
@@ -59,6 +60,8 @@ def lib() -> ctypes.CDLL:
             "moe_grouped_ffn": [sp, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp],
             "moe_layer_forward_routed": [sp, vp, vp, vp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp],
             "moe_selftest_wait_timeout": [sp, vp, i64, vp, vp, i64, vp, vp, sz, vp],
+            "moe_select_top_p": [sp, vp, ctypes.c_float, vp, vp, vp, vp],
+            "moe_select_rel_threshold": [sp, vp, ctypes.c_float, vp, vp, vp, vp],
             "moe_shared_ffn": [sp, vp, vp, vp, vp, vp, vp, sz, vp],
             "moe_combine": [sp, vp, vp, vp, vp, vp, vp, vp],
             "moe_layer_forward": [sp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, sz, vp],
@@ -205,6 +208,19 @@ def moe_selftest_wait_timeout(shape, expert_offsets, budget, W2, y_perm, wait_li
     _check("moe_selftest_wait_timeout",
            lib().moe_selftest_wait_timeout(ctypes.byref(shape), _p(expert_offsets), int(budget), _p(W2), _p(y_perm),
                                            int(wait_limit_clk), _p(dev_status), _p(ws), ws.numel(), _stream(stream)))
+
+
+def moe_select_top_p(shape, topk_score, P, n_sel, total, dev_status, stream=None):
+    """Top-P count per token (the Dynamic-MoE baseline); `total` (device int32 [1] or None) accumulates sum n_sel."""
+    _check("moe_select_top_p", lib().moe_select_top_p(ctypes.byref(shape), _p(topk_score), float(P), _p(n_sel),
+                                                      _p(total), _p(dev_status), _stream(stream)))
+
+
+def moe_select_rel_threshold(shape, topk_score, beta, n_sel, total, dev_status, stream=None):
+    """Skipping relative to the top-1 score (the NAEE baseline extended to Top-K)."""
+    _check("moe_select_rel_threshold",
+           lib().moe_select_rel_threshold(ctypes.byref(shape), _p(topk_score), float(beta), _p(n_sel), _p(total),
+                                          _p(dev_status), _stream(stream)))
 
 
 def moe_rmsnorm(shape, x, out, stream=None):

@@ -1,6 +1,7 @@
 // C-ABI entry points (see include/allocmoe.h): argument checks, workspace carve-up, launches.
 // Nothing here allocates or synchronises; every launch goes to the caller's stream.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include "allocmoe.h"
 
@@ -21,6 +22,7 @@ moe_status launch_moe_route(const moe_shape*, const float*, const int32_t*, int6
 moe_status launch_moe_combine(const moe_shape*, const uint16_t*, const int32_t*, const float*, const int32_t*,
                               const uint16_t*, const uint16_t*, long long, uint16_t*, cudaStream_t);
 moe_status launch_rmsnorm(const moe_shape*, const uint16_t*, uint16_t*, cudaStream_t);
+moe_status launch_token_rule_select(const moe_shape*, const float*, int, float, int32_t*, int32_t*, int32_t*, cudaStream_t);
 
 namespace {
 
@@ -64,6 +66,15 @@ WsLayout ws_layout(const moe_shape* s, int64_t budget_max) {
   return L;
 }
 
+// One NVTX range per C-ABI call (header-only NVTX: a no-op costing a few nanoseconds unless a profiler is
+// attached), so that a timeline shows which entry point enqueued which kernels.
+struct ApiRange {
+  explicit ApiRange(const char* name) { nvtxRangePushA(name); }
+  ~ApiRange() { nvtxRangePop(); }
+  ApiRange(const ApiRange&) = delete;
+  ApiRange& operator=(const ApiRange&) = delete;
+};
+
 template <typename T>
 T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<unsigned char*>(ws) + off); }
 
@@ -99,6 +110,7 @@ size_t moe_workspace_bytes(const moe_shape* shape, int64_t budget_max) {
 
 moe_status moe_gate(const moe_shape* shape, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,
                     float* scores, int32_t* topk_idx, float* topk_score, void* stream) {
+  ApiRange nvtx_range("moe_gate");
   if (!shape_ok(shape) || !x || !W_gate || !topk_idx || !topk_score) return MOE_ERR_ARG;
   if (!aligned16(x) || !aligned16(W_gate) || !aligned16(topk_idx) || !aligned16(topk_score)) return MOE_ERR_ARG;
   return launch_moe_gate(shape, x, W_gate, gate_bias, scores, topk_idx, topk_score, nullptr, 0, (cudaStream_t)stream);
@@ -106,6 +118,7 @@ moe_status moe_gate(const moe_shape* shape, const uint16_t* x, const uint16_t* W
 
 moe_status alloc_t_select(const moe_shape* shape, const float* topk_score, int64_t budget, int32_t* n_sel,
                           int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  ApiRange nvtx_range("alloc_t_select");
   (void)ws;
   (void)ws_bytes;
   if (!shape_ok(shape) || !topk_score || !n_sel || !dev_status) return MOE_ERR_ARG;
@@ -118,6 +131,7 @@ moe_status moe_permute(const moe_shape* shape, const uint16_t* x, const int32_t*
                        const int32_t* n_sel, int64_t budget, int32_t* expert_offsets, int32_t* perm_token,
                        float* perm_weight, int32_t* pair_pos, uint16_t* x_perm, int32_t* dev_status, void* ws,
                        size_t ws_bytes, void* stream) {
+  ApiRange nvtx_range("moe_permute");
   if (!shape_ok(shape) || !topk_idx || !topk_score || !n_sel || !expert_offsets || !perm_token || !perm_weight ||
       !pair_pos || !dev_status || !ws)
     return MOE_ERR_ARG;
@@ -133,6 +147,7 @@ moe_status moe_permute(const moe_shape* shape, const uint16_t* x, const int32_t*
 moe_status moe_route(const moe_shape* shape, const int32_t* topk_idx, const float* topk_score, int64_t budget,
                      int32_t* n_sel, int32_t* expert_offsets, int32_t* perm_token, float* perm_weight, int32_t* pair_pos,
                      int32_t* dev_status, void* stream) {
+  ApiRange nvtx_range("moe_route");
   if (!shape_ok(shape) || !topk_idx || !topk_score || !n_sel || !expert_offsets || !perm_token || !perm_weight ||
       !pair_pos || !dev_status)
     return MOE_ERR_ARG;
@@ -146,6 +161,7 @@ moe_status moe_route(const moe_shape* shape, const int32_t* topk_idx, const floa
 moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_or_xperm, const int32_t* perm_token,
                            const int32_t* expert_offsets, int64_t budget, const uint16_t* W13, const uint16_t* W2,
                            uint16_t* y_perm, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  ApiRange nvtx_range("moe_grouped_ffn");
   if (!shape_ok(shape) || !x_or_xperm || !expert_offsets || !W13 || !W2 || !y_perm || !dev_status || !ws)
     return MOE_ERR_ARG;
   if (!aligned16(x_or_xperm) || !aligned16(W13) || !aligned16(W2) || !aligned16(y_perm) || !aligned16(ws))
@@ -180,6 +196,7 @@ moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_or_xperm, c
 
 moe_status moe_shared_ffn(const moe_shape* shape, const uint16_t* x, const uint16_t* Wsh13, const uint16_t* Wsh2,
                           uint16_t* y_shared, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  ApiRange nvtx_range("moe_shared_ffn");
   if (!shape_ok(shape) || shape->S < 1 || !x || !Wsh13 || !Wsh2 || !y_shared || !dev_status || !ws) return MOE_ERR_ARG;
   if (!aligned16(x) || !aligned16(Wsh13) || !aligned16(Wsh2) || !aligned16(y_shared) || !aligned16(ws)) return MOE_ERR_ARG;
   const WsLayout L = ws_layout(shape, 0);
@@ -200,6 +217,7 @@ moe_status moe_shared_ffn(const moe_shape* shape, const uint16_t* x, const uint1
 moe_status moe_combine(const moe_shape* shape, const uint16_t* y_perm, const int32_t* pair_pos,
                        const float* topk_score, const int32_t* n_sel, const uint16_t* y_shared, uint16_t* out,
                        void* stream) {
+  ApiRange nvtx_range("moe_combine");
   if (!shape_ok(shape) || !y_perm || !pair_pos || !topk_score || !n_sel || !out) return MOE_ERR_ARG;
   if (!aligned16(y_perm) || !aligned16(out) || (y_shared && !aligned16(y_shared))) return MOE_ERR_ARG;
   return launch_moe_combine(shape, y_perm, pair_pos, topk_score, n_sel, y_shared, nullptr,
@@ -210,6 +228,7 @@ moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const ui
                              const uint16_t* W13, const uint16_t* W2, const uint16_t* Wsh13, const uint16_t* Wsh2,
                              int64_t budget, const uint16_t* residual, uint16_t* out, int32_t* dev_status, void* ws,
                              size_t ws_bytes, void* stream) {
+  ApiRange nvtx_range("moe_layer_forward");
   if (!shape_ok(shape) || !x || !W_gate || !W13 || !W2 || !out || !dev_status || !ws) return MOE_ERR_ARG;
   if (shape->S > 0 && (!Wsh13 || !Wsh2)) return MOE_ERR_ARG;
   if (!aligned16(x) || !aligned16(W_gate) || !aligned16(W13) || !aligned16(W2) || !aligned16(out) || !aligned16(ws))
@@ -290,6 +309,7 @@ moe_status moe_layer_forward_routed(const moe_shape* shape, const uint16_t* x, c
                                     int64_t budget_hint, const uint16_t* W13, const uint16_t* W2, const uint16_t* Wsh13,
                                     const uint16_t* Wsh2, const uint16_t* residual, uint16_t* out, int32_t* dev_status,
                                     void* ws, size_t ws_bytes, void* stream) {
+  ApiRange nvtx_range("moe_layer_forward_routed");
   if (!shape_ok(shape) || !x || !topk_idx || !topk_score || !n_sel || !W13 || !W2 || !out || !dev_status || !ws)
     return MOE_ERR_ARG;
   if (shape->S > 0 && (!Wsh13 || !Wsh2)) return MOE_ERR_ARG;
@@ -353,6 +373,7 @@ moe_status moe_layer_forward_routed(const moe_shape* shape, const uint16_t* x, c
 moe_status moe_selftest_wait_timeout(const moe_shape* shape, const int32_t* expert_offsets, int64_t budget,
                                      const uint16_t* W2, uint16_t* y_perm, int64_t wait_limit_clk, int32_t* dev_status,
                                      void* ws, size_t ws_bytes, void* stream) {
+  ApiRange nvtx_range("moe_selftest_wait_timeout");
   if (!shape_ok(shape) || !expert_offsets || !W2 || !y_perm || !dev_status || !ws) return MOE_ERR_ARG;
   if (!aligned16(W2) || !aligned16(y_perm) || !aligned16(ws)) return MOE_ERR_ARG;
   if (budget < 1 || budget > (int64_t)shape->K_orig * shape->T) return MOE_ERR_BUDGET;
@@ -376,7 +397,22 @@ moe_status moe_selftest_wait_timeout(const moe_shape* shape, const int32_t* expe
   return launch_ffn(a);
 }
 
+moe_status moe_select_top_p(const moe_shape* shape, const float* topk_score, float P, int32_t* n_sel, int32_t* total,
+                            int32_t* dev_status, void* stream) {
+  ApiRange nvtx_range("moe_select_top_p");
+  if (!shape_ok(shape) || !topk_score || !n_sel || !dev_status || !(P == P)) return MOE_ERR_ARG;
+  return launch_token_rule_select(shape, topk_score, 0, P, n_sel, total, dev_status, (cudaStream_t)stream);
+}
+
+moe_status moe_select_rel_threshold(const moe_shape* shape, const float* topk_score, float beta, int32_t* n_sel,
+                                    int32_t* total, int32_t* dev_status, void* stream) {
+  ApiRange nvtx_range("moe_select_rel_threshold");
+  if (!shape_ok(shape) || !topk_score || !n_sel || !dev_status || !(beta >= 0.f)) return MOE_ERR_ARG;
+  return launch_token_rule_select(shape, topk_score, 1, beta, n_sel, total, dev_status, (cudaStream_t)stream);
+}
+
 moe_status moe_rmsnorm(const moe_shape* shape, const uint16_t* x, uint16_t* out, void* stream) {
+  ApiRange nvtx_range("moe_rmsnorm");
   if (!shape_ok(shape) || !x || !out || !aligned16(x) || !aligned16(out)) return MOE_ERR_ARG;
   return launch_rmsnorm(shape, x, out, (cudaStream_t)stream);
 }

@@ -18,6 +18,20 @@ DEV void set_dev_status(int32_t* dev_status, moe_status s) {
   if (dev_status != nullptr) atomicOr(dev_status, 1 << (int)s);
 }
 
+// Values that index global memory and come from device data (expert_offsets, perm_token) are clamped to their
+// valid range before use, so that a list left behind by a routing step that reported an error cannot lead
+// outside the caller's buffers.  The checked build (-DALLOCMOE_CHECKED, `build.py --checked`) also reports every
+// value that needed clamping as MOE_ERR_ARG in the status word, which turns silent corruption upstream into an
+// error the caller sees.
+DEV int clamp_index(int v, int lo, int hi, int32_t* dev_status) {
+#ifdef ALLOCMOE_CHECKED
+  if (v < lo || v > hi) set_dev_status(dev_status, MOE_ERR_ARG);
+#else
+  (void)dev_status;
+#endif
+  return min(max(v, lo), hi);
+}
+
 DEV uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 // ------------------------------------------------------------------ programmatic dependent launch
@@ -195,6 +209,10 @@ DEV void tma_gather4_2d(void* smem_dst, const void* tmap, uint64_t* bar, int c0,
       ::"r"(smem_u32(smem_dst)), "l"((uint64_t)tmap), "r"(smem_u32(bar)), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
       : "memory");
 }
+
+// Orders this thread's earlier generic-proxy accesses to shared memory (ldmatrix reads of a ring slot, made
+// visible to it by a barrier) before async-proxy writes it issues afterwards (the TMA load that refills the slot).
+DEV void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ------------------------------------------------------------------ tcgen05 / TMEM
 DEV void tmem_alloc(uint32_t* smem_result, uint32_t ncols) {   // whole warp

@@ -107,7 +107,7 @@ DEV GatherRows gather_rows_of_tile(const FfnGemmParams& p, int a_row, int m_end,
     for (int i = 0; i < 4; ++i) {
       const int m = min(a_row + 4 * lane + i, p.gather_rows - 1);
       // clamped: a routing step that reported an error may leave anything in the list
-      g.r[i] = p.gather_idx != nullptr ? min(max(__ldg(p.gather_idx + m), 0), p.gather_src_rows - 1) : m;
+      g.r[i] = p.gather_idx != nullptr ? clamp_index(__ldg(p.gather_idx + m), 0, p.gather_src_rows - 1, p.dev_status) : m;
     }
   }
   return g;
@@ -260,8 +260,8 @@ ffn_gemm_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap tmA_r
   for (int gi = tid; gi < n_groups; gi += kFfnThreads) {
     if (gi < p.n_experts) {
       // clamped to the routed matrices' rows: a routing step that reported an error may leave anything here
-      const int lo = min(max(p.expert_offsets[gi], 0), p.routed_rows);
-      const int hi = min(max(p.expert_offsets[gi + 1], lo), p.routed_rows);
+      const int lo = clamp_index(p.expert_offsets[gi], 0, p.routed_rows, p.dev_status);
+      const int hi = clamp_index(p.expert_offsets[gi + 1], lo, p.routed_rows, p.dev_status);
       ctl->row_start[gi] = lo;
       ctl->row_count[gi] = hi - lo;
     } else {
@@ -541,8 +541,8 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
   for (int gi = tid; gi < n_groups; gi += kFfnThreads) {
     if (gi < p.n_experts) {
       // clamped to the routed matrices' rows: a routing step that reported an error may leave anything here
-      const int lo = min(max(p.expert_offsets[gi], 0), p.routed_rows);
-      const int hi = min(max(p.expert_offsets[gi + 1], lo), p.routed_rows);
+      const int lo = clamp_index(p.expert_offsets[gi], 0, p.routed_rows, p.dev_status);
+      const int hi = clamp_index(p.expert_offsets[gi + 1], lo, p.routed_rows, p.dev_status);
       ctl->row_start[gi] = lo;
       ctl->row_count[gi] = hi - lo;
     } else {
@@ -770,38 +770,7 @@ ffn_gemm_pair_kernel(const FfnGemmParams p, const __grid_constant__ CUtensorMap 
 using namespace allocmoe;
 
 // ------------------------------------------------------------------ host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (fn == nullptr) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      return nullptr;
-    fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
-// bf16 tensor [d2][d1][d0] (d0 contiguous), box {64, box1, 1}, 128-byte swizzle, zero fill.
-static bool make_tmap(CUtensorMap* tm, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1_elems,
-                      uint64_t stride2_elems, uint32_t box1) {
-  EncodeTiledFn fn = get_encode_fn();
-  if (fn == nullptr) return false;
-  cuuint64_t dims[3] = {d0, d1, d2};
-  cuuint64_t strides[2] = {stride1_elems * 2, stride2_elems * 2};
-  cuuint32_t box[3] = {(cuuint32_t)kBK, box1, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  const int rank = d2 > 0 ? 3 : 2;
-  if (rank == 2) dims[2] = 1;
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
+#include "tmap.h"
 
 // SM count of the current device (the persistent kernels' grid), looked up once per device.
 static PerDeviceInt g_num_sms;

@@ -111,6 +111,8 @@ moe_status launch_moe_permute(const moe_shape* s, const uint16_t* x, const int32
 // carries these 256 KB until the process exits.
 #include <mutex>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "shape_check.h"
 
 namespace {
@@ -142,6 +144,8 @@ extern "C" moe_status moe_permute_static(const moe_shape* shape, const uint16_t*
                                          const float* topk_score, const int32_t* n_sel, int64_t budget,
                                          int32_t* expert_offsets, int32_t* perm_token, float* perm_weight,
                                          int32_t* pair_pos, uint16_t* x_perm, int32_t* dev_status, void* stream) {
+  nvtxRangePushA("moe_permute_static");
+  struct Pop { ~Pop() { nvtxRangePop(); } } pop;
   const moe_shape* s = shape;
   if (!allocmoe::shape_ok(s)) return MOE_ERR_ARG;   // the same shapes as moe_permute accepts
   if (!topk_idx || !topk_score || !n_sel || !expert_offsets || !perm_token || !perm_weight || !pair_pos || !dev_status)

@@ -75,6 +75,77 @@ def test_alloc_t_select_flags_nonfinite_and_rejects_bad_budgets():
         assert ei.value.status == B.MOE_ERR_BUDGET
 
 
+# ----------------------------------------------------------------------------- Top-P / relative-threshold selection
+def _softmax_topk(T, N, K, seed):
+    g = torch.Generator().manual_seed(seed)
+    p = orc.softmax_scores((2.0 * torch.randn(T, N, generator=g, dtype=torch.float64)).numpy())
+    return orc.topk_sorted(p, K)
+
+
+@pytest.mark.parametrize("T,N,K", [(1, 8, 2), (64, 64, 6), (777, 16, 4), (4096, 64, 6), (5000, 128, 16)])
+def test_token_rule_selection_bit_exact(T, N, K):
+    """Top-P count and skipping relative to the top-1 score: n_sel equals the oracle's for every token (both take the
+    decision in fp32, columns in order), the kept total is their sum."""
+    _, sc = _softmax_topk(T, N, K, T + K)
+    sd = torch.from_numpy(sc).cuda()
+    shape = B.make_shape(T, 64, N, 64, 0, K, 1)
+    n_sel = torch.empty(T, dtype=torch.int32, device="cuda")
+    total = torch.zeros(1, dtype=torch.int32, device="cuda")
+    st = _status()
+    for P in (0.0, 0.05, 0.3, 0.5, float(sc[0, 0]), float(sc[0, :2].sum()), 0.8, 0.95, 1.5):
+        n_sel.fill_(-7)
+        total.zero_()
+        B.moe_select_top_p(shape, sd, P, n_sel, total, st)
+        torch.cuda.synchronize()
+        want = orc.top_p_count(sc, P)
+        assert np.array_equal(n_sel.cpu().numpy(), want), P
+        assert total.item() == int(want.sum())
+    for beta in (0.0, 0.01, 0.1, 0.25, 0.5, float(sc[0, 1] / sc[0, 0]), 1.0, 1.5):
+        n_sel.fill_(-7)
+        total.zero_()
+        B.moe_select_rel_threshold(shape, sd, beta, n_sel, total, st)
+        torch.cuda.synchronize()
+        want = orc.rel_threshold_count(sc, beta)
+        assert np.array_equal(n_sel.cpu().numpy(), want), beta
+        assert total.item() == int(want.sum())
+    assert st.item() == 0
+    bad = sd.clone()
+    bad[T // 2, 0] = float("inf")
+    B.moe_select_top_p(shape, bad, 0.5, n_sel, None, st)
+    torch.cuda.synchronize()
+    assert st.item() & (1 << B.MOE_ERR_NONFINITE)
+    assert ((n_sel >= 1) & (n_sel <= K)).all()
+
+
+def test_layer_runs_on_a_calibrated_top_p_selection():
+    """The comparison path end to end on a small layer: calibrate P so that the kept total meets the layer budget,
+    select, run moe_layer_forward_routed on that selection, compare with the oracle's Eq. 2 on the same counts."""
+    from paper_2604_08133_b200 import token_baselines as TB
+    cfg = synth.CONFIGS["c2"].with_(T=300, H=256, N=16, I=128, S=1, K_orig=4, K_base=1, budget=700)
+    d = synth.make_layer(cfg, device="cuda")
+    shape = B.shape_of(cfg)
+    idx = torch.empty(cfg.T, cfg.K_orig, dtype=torch.int32, device="cuda")
+    sc = torch.empty(cfg.T, cfg.K_orig, device="cuda")
+    B.moe_gate(shape, d["x"], d["W_gate"], d["gate_bias"], None, idx, sc)
+    st = _status()
+    for rule, inc, hi in (("top_p", True, 2.0), ("rel", False, 1.5)):
+        sel = TB.library_selector(rule, shape, st)
+        thr, tot = TB.calibrate(sel, sc, cfg.budget, increasing=inc, lo=0.0, hi=hi)
+        n_sel, tot2 = sel(sc, thr)
+        assert tot == tot2 and cfg.budget - cfg.T <= tot <= cfg.budget
+        want_n = (orc.top_p_count if rule == "top_p" else orc.rel_threshold_count)(sc.cpu().numpy(), thr)
+        assert np.array_equal(n_sel.cpu().numpy(), want_n)
+        ws = B.new_workspace(shape, cfg.budget)
+        out = torch.empty_like(d["x"])
+        B.moe_layer_forward_routed(shape, d["x"], idx, sc, n_sel, cfg.budget, tot, d["W13"], d["W2"], d["Wsh13"], d["Wsh2"],
+                                   out, st, ws)
+        torch.cuda.synchronize()
+        assert st.item() == 0
+        ref = orc.combine(np32(d["x"]), idx.cpu().numpy(), sc.cpu().numpy(), want_n, np32(d["W13"]), np32(d["W2"]),
+                          np32(d["Wsh13"]), np32(d["Wsh2"]))
+        assert max_rel(out.float().cpu().numpy(), ref) <= TOL_OUT
+
+
 # ----------------------------------------------------------------------------- moe_permute
 @pytest.mark.parametrize("T,N,K,kb,mult", [(64, 8, 2, 0, 1.0), (64, 64, 6, 1, 3.0), (1000, 64, 6, 1, 2.5),
                                             (4096, 64, 6, 1, 4.5), (4096, 64, 6, 1, 6.0), (777, 16, 4, 0, 1.3),
@@ -173,7 +244,11 @@ def test_moe_permute_flags_a_count_mismatch():
 
 # ----------------------------------------------------------------------------- moe_gate
 @pytest.mark.parametrize("name,kw", [("c1", {}), ("c2", {}), ("c2", dict(T=333, H=192, N=24, K_orig=5)),
-                                      ("c3", dict(T=1000)), ("c5", dict(T=500))])
+                                      ("c3", dict(T=1000)), ("c5", dict(T=500)),
+                                      # large batches: ragged last tile, a 64-wide last chunk of H, N = 128, a full
+                                      # prefill batch
+                                      ("c3", dict(T=1100, H=192)), ("c3", dict(T=1030, H=1024, N=128, K_orig=16)),
+                                      ("c3", dict(T=4096)), ("c5", dict(T=1500))])
 def test_moe_gate_against_oracle(name, kw):
     cfg = synth.CONFIGS[name].with_(I=64, S=0, **kw)
     x = synth.normal_bf16((cfg.T, cfg.H), 1.0, synth.stream_key(cfg.seed, 0, 0))
@@ -386,6 +461,46 @@ def test_bounded_wait_runs_out_and_the_kernel_returns(T, budget):
     assert max_rel(y[offn[e]:offn[e + 1]].float().cpu().numpy(), want) <= TOL_OUT
     with pytest.raises(B.MoeError):
         B.moe_selftest_wait_timeout(shape, off, budget, W2, y, 10, st, ws)         # limit below the accepted range
+
+
+def test_checked_build_reports_clamped_indices():
+    """The -DALLOCMOE_CHECKED build of the library gives the same results and additionally raises MOE_ERR_ARG when an
+    expert offset or a token index had to be clamped into range.  Runs in a process of its own (another .so)."""
+    import os
+    import subprocess
+    import sys
+    from paper_2604_08133_b200 import build as bld
+    lib = bld.build(checked=True)
+    code = r"""
+import numpy as np, torch
+from paper_2604_08133_b200 import binding as B, synth
+assert B.LIB_PATH.endswith("liballocmoe_checked.so")
+T, H, N, I = 300, 128, 8, 128
+cfg = synth.CONFIGS["c1"].with_(T=T, H=H, N=N, I=I)
+d = synth.make_layer(cfg, device="cuda")
+shape = B.shape_of(cfg); ws = B.new_workspace(shape, T)
+st = torch.zeros(1, dtype=torch.int32, device="cuda")
+good = torch.tensor([0, 100, 100, 100, 260, 260, 260, 260, 300], dtype=torch.int32).cuda()
+tok = torch.arange(T, dtype=torch.int32).cuda()
+y0 = torch.empty(T, H, dtype=torch.bfloat16, device="cuda"); y1 = torch.empty_like(y0)
+B.moe_grouped_ffn(shape, d["x"], None, good, T, d["W13"], d["W2"], y0, st, ws)
+B.moe_grouped_ffn(shape, d["x"], tok, good, T, d["W13"], d["W2"], y1, st, ws)
+torch.cuda.synchronize()
+assert st.item() == 0 and torch.equal(y0, y1)
+bad = torch.tensor([0, 100, 100, 100, 260, 260, 260, 260, 10 ** 6], dtype=torch.int32).cuda()
+B.moe_grouped_ffn(shape, d["x"], None, bad, T, d["W13"], d["W2"], y1, st, ws)
+torch.cuda.synchronize()
+assert st.item() == 1 << B.MOE_ERR_ARG, st.item()
+st.zero_(); tok[7] = -3
+B.moe_grouped_ffn(shape, d["x"], tok, good, T, d["W13"], d["W2"], y1, st, ws)
+torch.cuda.synchronize()
+assert st.item() == 1 << B.MOE_ERR_ARG, st.item()
+print("checked ok")
+"""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", code], env=dict(os.environ, ALLOCMOE_LIB=lib, PYTHONPATH=root),
+                       capture_output=True, text=True, timeout=600, cwd=root)
+    assert r.returncode == 0 and "checked ok" in r.stdout, r.stdout[-1500:] + r.stderr[-1500:]
 
 
 @pytest.mark.parametrize("pair,gather,tile_n", [("0", "0", "256"), ("1", "0", "256"), ("0", "1000000", "256"),
