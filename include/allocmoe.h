@@ -72,7 +72,10 @@ size_t moe_workspace_bytes(const moe_shape* shape, int64_t budget_max);
  *   gate_bias  device fp32 [N] or NULL: added to the logits before the softmax
  *   scores     device fp32 [T,N] or NULL (full softmax output, optional)
  *   topk_idx   device int32 [T,K_orig]
- *   topk_score device fp32 [T,K_orig] */
+ *   topk_score device fp32 [T,K_orig]
+ * From about a thousand tokens on, with 64 or 128 experts, the contraction runs on the tensor cores fed by TMA; its
+ * waits are bounded, and should one run out the affected tokens' scores are written as NaN (alloc_t_select then
+ * reports MOE_ERR_NONFINITE; inside moe_layer_forward MOE_ERR_TIMEOUT is raised as well). */
 moe_status moe_gate(const moe_shape* shape, const uint16_t* x, const uint16_t* W_gate,
                     const float* gate_bias, float* scores, int32_t* topk_idx, float* topk_score,
                     void* stream);

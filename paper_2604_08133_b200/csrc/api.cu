@@ -10,7 +10,7 @@
 
 // launchers defined next to their kernels
 moe_status launch_moe_gate(const moe_shape*, const uint16_t*, const uint16_t*, const float*, float*, int32_t*, float*,
-                           int32_t*, int, cudaStream_t);
+                           int32_t*, int, int32_t*, cudaStream_t);
 moe_status launch_alloc_t_select(const moe_shape*, const float*, int64_t, int32_t*, int32_t*, cudaStream_t);
 moe_status launch_moe_permute(const moe_shape*, const uint16_t*, const int32_t*, const float*, const int32_t*, int64_t,
                               int32_t*, int32_t*, float*, int32_t*, uint16_t*, int32_t*, int32_t*, bool, cudaStream_t);
@@ -113,7 +113,8 @@ moe_status moe_gate(const moe_shape* shape, const uint16_t* x, const uint16_t* W
   ApiRange nvtx_range("moe_gate");
   if (!shape_ok(shape) || !x || !W_gate || !topk_idx || !topk_score) return MOE_ERR_ARG;
   if (!aligned16(x) || !aligned16(W_gate) || !aligned16(topk_idx) || !aligned16(topk_score)) return MOE_ERR_ARG;
-  return launch_moe_gate(shape, x, W_gate, gate_bias, scores, topk_idx, topk_score, nullptr, 0, (cudaStream_t)stream);
+  return launch_moe_gate(shape, x, W_gate, gate_bias, scores, topk_idx, topk_score, nullptr, 0, nullptr,
+                         (cudaStream_t)stream);
 }
 
 moe_status alloc_t_select(const moe_shape* shape, const float* topk_score, int64_t budget, int32_t* n_sel,
@@ -256,7 +257,7 @@ moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const ui
   prof_mark(0, st);
   // the gate launch also clears the expert GEMMs' row-block counters (no memset between kernels of the call)
   moe_status r = launch_moe_gate(shape, x, W_gate, gate_bias, nullptr, topk_idx, topk_score, at<int32_t>(ws, L.gemm_done),
-                                 (int)ffn_done_ints(shape, budget), st);
+                                 (int)ffn_done_ints(shape, budget), dev_status, st);
   if (r != MOE_OK) return r;
   prof_mark(1, st);
   if (moe_route_fits(shape)) {

@@ -14,6 +14,7 @@
 #include <cooperative_groups.h>
 
 #include "common.cuh"
+#include "tmap.h"
 
 namespace cg = cooperative_groups;
 
@@ -232,6 +233,181 @@ moe_gate_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __rest
   cluster.sync();   // no CTA leaves while a peer may still read its partial sums
 }
 
+// ------------------------------------------------------------------------------------------------
+// Large batches (about a thousand tokens and more) with N = 64 or 128 experts: the contraction on the
+// 5th-generation tensor cores.  On B200 the mma.sync path above tops out near 190 TFLOP/s for the whole
+// GPU, which made the kernel above compute-bound on 4096 tokens (17 us however its chunks were loaded:
+// cp.async, per-row bulk copies and TMA boxes all measured the same); tcgen05.mma removes that bound.
+//
+// Same decomposition: a cluster of KS CTAs per token tile (128 tokens here = UMMA M), rank r taking 64-wide
+// blocks r, r + KS, ... of H, partial logits added in rank order through distributed shared memory, then
+// gate_finish.  Per block one TMA box of x (128 tokens x 64, K-major, the A operand) and one box per 64
+// experts of W_gate (64 rows of H x 64 experts: N-contiguous, i.e. an MN-major B operand, which the
+// instruction descriptor's B-major bit and the shared-memory descriptor below express: 8-row groups along K
+// are 1024 bytes apart, 64-expert blocks one box apart), all written with the 128-byte swizzle.  A CTA's
+// blocks (at most 8) all have their own stage, so every load is issued up front and no stage is reused.
+// One thread issues the loads and the MMAs (M = 128, N = 64 or 128, K = 16; fp32 accumulator in TMEM); then
+// all eight warps read the accumulator (warp w: lanes 32 (w % 4).., half of the columns each) into shared
+// memory for the cluster-wide reduction.
+//
+// Waits are bounded.  A wait that runs out marks the tile's scores NaN (which the selection reports as
+// MOE_ERR_NONFINITE) and raises MOE_ERR_TIMEOUT in dev_status when the caller gave one; the CTA still takes
+// part in every cluster barrier, waits for its copies in flight and frees its tensor memory before it exits.
+constexpr int kUGateTM = 128;
+constexpr int kUGateBK = 64;
+constexpr int kUGateMaxStages = 8;
+constexpr int kUGateXBytes = kUGateTM * kUGateBK * 2;      // 16 KB
+constexpr int kUGateWBoxBytes = kUGateBK * 64 * 2;         // 8 KB per 64 experts
+
+// MN-major operand, 128-byte swizzle: rows of 64 elements along N (128 bytes) per K index, groups of eight K
+// rows 1024 bytes apart (stride byte offset), 64-element blocks along N `n_block_bytes` apart (leading byte
+// offset).  Advancing 16 along K adds 2048 bytes to the start address.
+DEV uint64_t umma_desc_mn_sw128(uint32_t smem_addr, uint32_t n_block_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
+  d |= (uint64_t)((n_block_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+template <int NB64>   // N = 64 * NB64
+__global__ void __launch_bounds__(256, 1)
+moe_gate_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+                     const float* __restrict__ gate_bias, int T, int H, int N, int K_orig,
+                     float* __restrict__ scores, int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
+                     int32_t* __restrict__ zero_ptr, int zero_n, int32_t* dev_status) {
+  cg::cluster_group cluster = cg::this_cluster();
+  const int KS = (int)cluster.num_blocks();
+  const int ks_rank = (int)cluster.block_rank();
+  constexpr int NP = 64 * NB64, NW = 8, kThreads = 256;
+  constexpr int kStageBytes = kUGateXBytes + NB64 * kUGateWBoxBytes;
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  __shared__ uint64_t full[kUGateMaxStages];
+  __shared__ uint64_t acc_done;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int t0 = blockIdx.x * kUGateTM;
+  const int nblocks_all = (H + kUGateBK - 1) / kUGateBK;
+  const int nblocks = (nblocks_all - ks_rank + KS - 1) / KS;   // this CTA's blocks of H: ks_rank, ks_rank + KS, ... (<= 8)
+  if (tid == 0) {
+    for (int i = 0; i < kUGateMaxStages; ++i) mbar_init(&full[i], 1);
+    mbar_init(&acc_done, 1);
+    s_abort = 0;
+    fence_barrier_init();
+    prefetch_tensormap(&tm_x);
+    prefetch_tensormap(&tm_w);
+  }
+  if (warp == 1) {
+    tmem_alloc(&s_tmem, NP);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = s_tmem;
+  pdl_prologue_done();
+  if (zero_ptr != nullptr && blockIdx.x == 0 && blockIdx.y == 0)      // see moe_gate_kernel
+    for (int i = tid; i < zero_n; i += kThreads) zero_ptr[i] = 0;
+
+  if (tid == 0) {
+    // every block of this CTA has its own stage: all loads go out at once (columns past H and rows past T read as zero)
+    for (int b = 0; b < nblocks; ++b) {
+      const int k0 = (ks_rank + b * KS) * kUGateBK;
+      unsigned char* st = ring + b * kStageBytes;
+      mbar_expect_tx(&full[b], (uint32_t)kStageBytes);
+      tma_load_2d(st, &tm_x, &full[b], k0, t0);
+#pragma unroll
+      for (int nb = 0; nb < NB64; ++nb) tma_load_2d(st + kUGateXBytes + nb * kUGateWBoxBytes, &tm_w, &full[b], nb * 64, k0);
+    }
+    // instruction descriptor: fp32 accumulator, bf16 A and B, A K-major, B MN-major (bit 16)
+    constexpr uint32_t idesc = umma_idesc_bf16(kUGateTM, NP) | (1u << 16);
+    bool ok = true;
+    for (int b = 0; b < nblocks && ok; ++b) {
+      {   // bounded wait for the block's stage
+        if (!mbar_try_wait(&full[b], 0u)) {
+          const long long t_start = clock64();
+          while (!mbar_try_wait(&full[b], 0u))
+            if (clock64() - t_start > kWaitLimitClk) { ok = false; break; }
+        }
+      }
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t sa = smem_u32(ring + b * kStageBytes);
+      const uint64_t da = umma_desc_sw128(sa);
+      const uint64_t db = umma_desc_mn_sw128(sa + kUGateXBytes, (uint32_t)kUGateWBoxBytes);
+#pragma unroll
+      for (int k = 0; k < kUGateBK / 16; ++k)
+        umma_bf16(tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * (2048 >> 4)), idesc, (b | k) != 0 ? 1u : 0u);
+    }
+    if (!ok) s_abort = 1;
+    umma_commit(&acc_done);      // arrives once every MMA issued above has completed (at once if there were none)
+  }
+  __syncwarp();
+  // every warp: wait for the accumulator (bounded; lane 0 polls)
+  {
+    int ok = 1;
+    if (lane == 0 && !mbar_try_wait(&acc_done, 0u)) {
+      const long long t_start = clock64();
+      while (!mbar_try_wait(&acc_done, 0u)) {
+        __nanosleep(32);
+        if (clock64() - t_start > 2 * kWaitLimitClk) { ok = 0; break; }
+      }
+    }
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    if (!ok) s_abort = 1;
+  }
+  tc_fence_after_sync();
+  __syncthreads();   // s_abort is final; the MMAs no longer read the stages, which red[] aliases below
+  const bool aborted = s_abort != 0;
+
+  // partial logits to shared memory: red[row][col], fp32.  Warp w reads TMEM lanes 32 (w % 4) .. + 31 (= token rows)
+  // and the column half w / 4.
+  float* red = reinterpret_cast<float*>(ring);
+  constexpr int RS = NP + 1;
+  if (!aborted) {
+    const int q = warp & 3, half = warp >> 2;
+    const int row = q * 32 + lane;
+    constexpr int kColsPerWarp = NP / 2;
+#pragma unroll
+    for (int c = 0; c < kColsPerWarp / 32; ++c) {
+      uint32_t v[32];
+      const int col0 = half * kColsPerWarp + c * 32;
+      tmem_ld_32x32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)col0, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 32; ++i) red[row * RS + col0 + i] = __uint_as_float(v[i]);
+    }
+  } else {   // NaN partial sums give NaN scores in every CTA of the cluster
+    if (tid == 0) {
+      for (int b = 0; b < nblocks; ++b) mbar_wait_drain(&full[b], 0u);   // copies still in flight land first
+      set_dev_status(dev_status, MOE_ERR_TIMEOUT);
+    }
+    __syncthreads();
+    for (int i = tid; i < kUGateTM * RS; i += kThreads) red[i] = __int_as_float(0x7fc00000);
+  }
+  tc_fence_before_sync();
+  cluster.sync();   // every CTA's partial logits are in its red[0 .. 128*RS)
+
+  const float* rred[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) rred[k] = cluster.map_shared_rank(red, k < KS ? k : 0);
+  if (kUGateTM / KS >= NW * 4)
+    gate_finish<NP, NW, 8>(rred, KS, ks_rank, t0, T, N, K_orig, gate_bias, scores, topk_idx, topk_score);
+  else if (kUGateTM / KS >= NW * 2)
+    gate_finish<NP, NW, 16>(rred, KS, ks_rank, t0, T, N, K_orig, gate_bias, scores, topk_idx, topk_score);
+  else
+    gate_finish<NP, NW, 32>(rred, KS, ks_rank, t0, T, N, K_orig, gate_bias, scores, topk_idx, topk_score);
+  cluster.sync();   // no CTA leaves while a peer may still read its partial sums
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem, NP);
+  }
+}
+
 }  // namespace allocmoe
 
 using namespace allocmoe;
@@ -266,29 +442,85 @@ static moe_status gate_launch_t(const moe_shape* s, const uint16_t* x, const uin
   return err == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
+// The tcgen05 kernel.  KS: enough CTAs per 128-token tile that each holds at most kUGateMaxStages blocks of H and
+// the grid is about one CTA per SM.  False when the shape does not fit (the caller falls back to mma.sync).
+static bool gate_umma_fits(const moe_shape* s, int* ks_out) {
+  if (s->T < 1024 || (s->N != 64 && s->N != 128)) return false;
+  const int nblocks = (s->H + kUGateBK - 1) / kUGateBK;
+  const int stage = kUGateXBytes + (s->N / 64) * kUGateWBoxBytes;
+  const int max_stages = (200 * 1024) / stage < kUGateMaxStages ? (200 * 1024) / stage : kUGateMaxStages;
+  const int tiles = (s->T + kUGateTM - 1) / kUGateTM;
+  int ks = 1;
+  while ((nblocks + ks - 1) / ks > max_stages && ks < 8) ks *= 2;
+  if ((nblocks + ks - 1) / ks > max_stages) return false;
+  while (ks * 2 <= 8 && ks * 2 <= nblocks && tiles * ks * 2 <= 300) ks *= 2;
+  *ks_out = ks;
+  return true;
+}
+
+template <int NB64>
+static moe_status gate_launch_umma(const moe_shape* s, int ks, const uint16_t* x, const uint16_t* W_gate,
+                                   const float* gate_bias, float* scores, int32_t* topk_idx, float* topk_score,
+                                   int32_t* zero_ptr, int zero_n, int32_t* dev_status, cudaStream_t stream) {
+  constexpr int NP = 64 * NB64;
+  const int nblocks = (s->H + kUGateBK - 1) / kUGateBK;
+  const int per_cta = (nblocks + ks - 1) / ks;
+  const size_t stage = (size_t)kUGateXBytes + (size_t)NB64 * kUGateWBoxBytes;
+  size_t smem = per_cta * stage;
+  const size_t red = (size_t)kUGateTM * (NP + 1) * 4;
+  if (smem < red) smem = red;
+  smem += 1024;   // the stages start on a 1024-byte boundary (swizzle pattern)
+  CUtensorMap tm_x, tm_w;
+  if (!make_tmap(&tm_x, x, (uint64_t)s->H, (uint64_t)s->T, 0, (uint64_t)s->H, 0, kUGateTM) ||
+      !make_tmap(&tm_w, W_gate, (uint64_t)s->N, (uint64_t)s->H, 0, (uint64_t)s->N, 0, kUGateBK))
+    return MOE_ERR_CUDA;
+  static PerDeviceOnce attr_set;
+  if (!ensure_dynamic_smem(moe_gate_umma_kernel<NB64>, 202 * 1024, attr_set)) return MOE_ERR_CUDA;
+  const int tiles = (s->T + kUGateTM - 1) / kUGateTM;
+  const cudaError_t err = launch_dependent(
+      moe_gate_umma_kernel<NB64>, dim3((unsigned)tiles, (unsigned)ks, 1), dim3(256), smem, stream, (unsigned)ks, tm_x, tm_w,
+      gate_bias, (int)s->T, (int)s->H, (int)s->N, (int)s->K_orig, scores, topk_idx, topk_score, zero_ptr, zero_n,
+      dev_status);
+  return err == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
 template <int NT16>
 static moe_status gate_launch_nw(const moe_shape* s, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,
                                  float* scores, int32_t* topk_idx, float* topk_score, int32_t* zero_ptr, int zero_n,
-                                 cudaStream_t stream) {
+                                 int32_t* dev_status, cudaStream_t stream) {
+  if constexpr (NT16 == 4 || NT16 == 8) {
+    int ks = 1;
+    if (gate_umma_fits(s, &ks))
+      return gate_launch_umma<NT16 / 4>(s, ks, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n,
+                                        dev_status, stream);
+  }
   if (s->T >= 2048)
     return gate_launch_t<NT16, 4>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
   return gate_launch_t<NT16, 2>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
 }
 
-// zero_ptr / zero_n: device ints the launch also clears (nullptr: none)
+// zero_ptr / zero_n: device ints the launch also clears (nullptr: none); dev_status: optional status word
 moe_status launch_moe_gate(const moe_shape* s, const uint16_t* x, const uint16_t* W_gate, const float* gate_bias,
                            float* scores, int32_t* topk_idx, float* topk_score, int32_t* zero_ptr, int zero_n,
-                           cudaStream_t stream) {
+                           int32_t* dev_status, cudaStream_t stream) {
   const int nt16 = (s->N + 15) / 16;
   switch (nt16) {
-    case 1: return gate_launch_nw<1>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
-    case 2: return gate_launch_nw<2>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
-    case 3: return gate_launch_nw<3>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
-    case 4: return gate_launch_nw<4>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
-    case 5: return gate_launch_nw<5>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
-    case 6: return gate_launch_nw<6>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
-    case 7: return gate_launch_nw<7>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
-    case 8: return gate_launch_nw<8>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, stream);
+    case 1: return gate_launch_nw<1>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, dev_status,
+                                     stream);
+    case 2: return gate_launch_nw<2>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, dev_status,
+                                     stream);
+    case 3: return gate_launch_nw<3>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, dev_status,
+                                     stream);
+    case 4: return gate_launch_nw<4>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, dev_status,
+                                     stream);
+    case 5: return gate_launch_nw<5>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, dev_status,
+                                     stream);
+    case 6: return gate_launch_nw<6>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, dev_status,
+                                     stream);
+    case 7: return gate_launch_nw<7>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, dev_status,
+                                     stream);
+    case 8: return gate_launch_nw<8>(s, x, W_gate, gate_bias, scores, topk_idx, topk_score, zero_ptr, zero_n, dev_status,
+                                     stream);
     default: return MOE_ERR_ARG;
   }
 }
