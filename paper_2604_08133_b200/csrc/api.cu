@@ -15,7 +15,7 @@ moe_status launch_alloc_t_select(const moe_shape*, const float*, int64_t, int32_
 moe_status launch_moe_permute(const moe_shape*, const uint16_t*, const int32_t*, const float*, const int32_t*, int64_t,
                               int32_t*, int32_t*, float*, int32_t*, uint16_t*, int32_t*, int32_t*, bool, cudaStream_t);
 moe_status launch_gather_rows(const moe_shape*, const uint16_t*, const int32_t*, int64_t, const int32_t*, uint16_t*,
-                              cudaStream_t);
+                              int32_t*, cudaStream_t);
 bool moe_route_fits(const moe_shape*);
 moe_status launch_moe_route(const moe_shape*, const float*, const int32_t*, int64_t, bool, int32_t*, int32_t*, int32_t*,
                             float*, int32_t*, int32_t*, cudaStream_t);
@@ -178,7 +178,7 @@ moe_status moe_grouped_ffn(const moe_shape* shape, const uint16_t* x_or_xperm, c
   if (perm_token != nullptr && budget > 0 && !ffn_gathers(shape, budget)) {
     // long expert runs: one copy of the rows into the workspace, then 128-row box loads, is faster than
     // fetching every tile's rows four at a time
-    const moe_status r = launch_gather_rows(shape, x_or_xperm, perm_token, budget, nullptr, at<uint16_t>(ws, L.x_perm), st);
+    const moe_status r = launch_gather_rows(shape, x_or_xperm, perm_token, budget, nullptr, at<uint16_t>(ws, L.x_perm), dev_status, st);
     if (r != MOE_OK) return r;
     a.a_routed = at<uint16_t>(ws, L.x_perm);
     a.gather_idx = nullptr;
@@ -266,7 +266,7 @@ moe_status moe_layer_forward(const moe_shape* shape, const uint16_t* x, const ui
                          pair_pos, dev_status, st);
     if (r != MOE_OK) return r;
     prof_mark(2, st);
-    if (budget > 0 && x_perm != nullptr) r = launch_gather_rows(shape, x, perm_token, budget, nullptr, x_perm, st);
+    if (budget > 0 && x_perm != nullptr) r = launch_gather_rows(shape, x, perm_token, budget, nullptr, x_perm, dev_status, st);
   } else {
     r = launch_alloc_t_select(shape, topk_score, budget, n_sel, dev_status, st);
     if (r != MOE_OK) return r;
@@ -341,7 +341,7 @@ moe_status moe_layer_forward_routed(const moe_shape* shape, const uint16_t* x, c
                          perm_token, perm_weight, pair_pos, dev_status, st);
     if (r != MOE_OK) return r;
     if (budget_max > 0 && x_perm != nullptr)
-      r = launch_gather_rows(shape, x, perm_token, budget_max, expert_offsets + shape->N, x_perm, st);
+      r = launch_gather_rows(shape, x, perm_token, budget_max, expert_offsets + shape->N, x_perm, dev_status, st);
   } else {
     r = launch_moe_permute(shape, x, topk_idx, topk_score, n_sel, budget_max, expert_offsets, perm_token, perm_weight,
                            pair_pos, x_perm, dev_status, at<int32_t>(ws, L.seg_counts), false, st);

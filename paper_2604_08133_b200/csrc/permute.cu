@@ -54,12 +54,11 @@ permute_place_kernel(const int32_t* __restrict__ topk_idx, const float* __restri
 // the list's length as the device knows it (expert_offsets[N]) when `rows` is only an upper bound.
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ perm_token, int T, int row_vec,
-                   long long rows, const int32_t* __restrict__ rows_dev, uint4* __restrict__ x_perm) {
+                   long long rows, const int32_t* __restrict__ rows_dev, uint4* __restrict__ x_perm, int32_t* dev_status) {
   pdl_prologue_done();
   if (rows_dev != nullptr) rows = min(rows, (long long)max(*rows_dev, 0));
   for (long long p = blockIdx.x; p < rows; p += gridDim.x) {
-    int t = perm_token[p];
-    t = min(max(t, 0), T - 1);
+    const int t = clamp_index(perm_token[p], 0, T - 1, dev_status);
     const uint4* src = x + (long long)t * row_vec;
     uint4* dst = x_perm + p * row_vec;
     for (int c = threadIdx.x; c < row_vec; c += blockDim.x) dst[c] = __ldg(src + c);
@@ -71,12 +70,12 @@ gather_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ perm
 using namespace allocmoe;
 
 moe_status launch_gather_rows(const moe_shape* s, const uint16_t* x, const int32_t* perm_token, int64_t budget,
-                              const int32_t* rows_dev, uint16_t* x_perm, cudaStream_t stream) {
+                              const int32_t* rows_dev, uint16_t* x_perm, int32_t* dev_status, cudaStream_t stream) {
   const int row_vec = s->H / 8;
   const long long g = budget < (1ll << 20) ? budget : (1ll << 20);
   return launch_dependent(gather_rows_kernel, dim3((unsigned)g), dim3(256), 0, stream, 1, reinterpret_cast<const uint4*>(x),
                           perm_token, (int)s->T, row_vec, (long long)budget, rows_dev,
-                          reinterpret_cast<uint4*>(x_perm)) == cudaSuccess
+                          reinterpret_cast<uint4*>(x_perm), dev_status) == cudaSuccess
              ? MOE_OK
              : MOE_ERR_CUDA;
 }
@@ -99,7 +98,7 @@ moe_status launch_moe_permute(const moe_shape* s, const uint16_t* x, const int32
                               pair_pos) == cudaSuccess;
   if (!ok) return MOE_ERR_CUDA;
   if (x_perm != nullptr && budget > 0)
-    return launch_gather_rows(s, x, perm_token, budget, exact ? nullptr : expert_offsets + s->N, x_perm, stream);
+    return launch_gather_rows(s, x, perm_token, budget, exact ? nullptr : expert_offsets + s->N, x_perm, dev_status, stream);
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
