@@ -91,6 +91,9 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the stage profile / full-Top-K / e2e passes")
     ap.add_argument("--no-workloads", action="store_true", help="headline workload only (no c3 / c5 / c4 entries)")
+    ap.add_argument("--blocks", type=int, default=None,
+                    help="time exactly this many blocks of --steps steps instead of repeating blocks to half a second "
+                         "(short runs for a profiler; such a run's numbers are not benchmark figures)")
     ap.add_argument("--global-alloc-t", action="store_true",
                     help="also time the batch-wide Alloc-T path (gate, all-gather of the score rows, selection over "
                          "the whole pool, routed layer call); always on with more than one GPU")
@@ -288,10 +291,11 @@ SECONDARY = (("c3", None), ("c5", None), ("c4", None))     # (workload, budget m
 class Env:
     """Process-group facts and the timing primitives shared by every measurement of a run."""
 
-    def __init__(self):
+    def __init__(self, blocks=None):
         import torch
         import torch.distributed as dist
         self.torch, self.dist = torch, dist
+        self.blocks = blocks
         self.world = int(os.environ.get("WORLD_SIZE", "1"))
         self.rank = int(os.environ.get("RANK", "0"))
         self.local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -324,6 +328,8 @@ class Env:
         first = one()
         n = max(MIN_BLOCKS, int(math.ceil(MIN_REGION_S * 1e3 / max(first, 1e-3))))
         n = min(n, MAX_BLOCKS)
+        if self.blocks is not None:
+            n = max(1, self.blocks)
         ms = [first] + [one() for _ in range(n - 1)]
         return [m / k for m in ms]
 
@@ -655,7 +661,7 @@ def parity_on_sample(cfg, budget, ref):
 def run_ours(args):
     import torch
     from paper_2604_08133_b200 import binding as B
-    env = Env()
+    env = Env(args.blocks)
     B.lib()   # fails loudly when the CUDA library is missing
 
     res = bench_workload(env, args, args.workload, args.budget_mult, args.steps, args.warmup, full=True)

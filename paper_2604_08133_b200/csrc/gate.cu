@@ -453,7 +453,7 @@ static bool gate_umma_fits(const moe_shape* s, int* ks_out) {
   int ks = 1;
   while ((nblocks + ks - 1) / ks > max_stages && ks < 8) ks *= 2;
   if ((nblocks + ks - 1) / ks > max_stages) return false;
-  while (ks * 2 <= 8 && ks * 2 <= nblocks && tiles * ks * 2 <= 300) ks *= 2;
+  while (ks * 2 <= 8 && ks * 2 <= nblocks && tiles * ks * 2 <= 160) ks *= 2;   // about one CTA per SM
   *ks_out = ks;
   return true;
 }
