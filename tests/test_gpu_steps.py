@@ -21,7 +21,12 @@ SELECT_CASES = [
     (1, 2, 1, None, False), (31, 3, 0, None, True), (64, 2, 0, None, False), (64, 6, 1, None, False),
     (1000, 6, 1, None, True), (1025, 4, 2, None, False), (4096, 6, 1, None, False), (4096, 6, 1, None, True),
     (4096, 6, 0, None, False), (2048, 6, 1, None, False), (8192, 2, 1, None, False), (8192, 8, 1, None, True),
-    (20000, 6, 1, None, False),      # pool of 100 000 keys: beyond the shared-memory staging
+    (20000, 6, 1, None, False),      # pool of 100 000 keys: beyond one CTA's shared memory -> a cluster of 3 CTAs
+    (32768, 6, 1, None, True),       # 8 ranks x 4096 tokens pooled (163 840 keys, many ties): a cluster of 5 CTAs
+    (32768, 6, 1, None, False),
+    (9001, 6, 0, None, True),        # 54 006 keys on 2 CTAs, an odd split of the tokens
+    (65536, 6, 1, [65536, 65537, 100000, 196608, 393215, 393216], True),   # 327 680 keys: the largest cluster, 8 CTAs
+    (70000, 6, 0, [0, 1, 140000, 420000], True),   # 420 000 keys: beyond the cluster too, one CTA re-reading L2
 ]
 
 
