@@ -221,6 +221,16 @@ def test_c5_large_experts_full_size():
     _sampled_check(cfg, d, cfg.budget, key=5)
 
 
+@pytest.mark.parametrize("name", ["qwen", "olmoe"])
+def test_other_model_shapes_full_size(name):
+    """The Qwen1.5-MoE-shaped (60 experts, Top-4, one shared expert) and OLMoE-shaped (64 experts, Top-8) prefill
+    layers at their benchmark size: routing in full, outputs on a tile-covering token sample."""
+    cfg = synth.CONFIGS[name]
+    d = dev_layer(cfg)
+    _, inter, _ = _sampled_check(cfg, d, cfg.budget, key=60 if name == "qwen" else 64)
+    assert int(inter["expert_offsets"][-1]) == cfg.budget
+
+
 def test_layer_beyond_8192_tokens_takes_the_unfused_routing_path():
     """Above 8192 tokens moe_layer_forward runs alloc_t_select and moe_permute's kernels one after the other instead
     of the one-launch routing step; small H and I keep the oracle's whole-layer run short."""
