@@ -75,6 +75,33 @@ def test_ragged_multi_tile_layer():
     _full_check(cfg)
 
 
+@pytest.mark.parametrize("S,T", [(1, 70), (0, 70), (2, 1500)])
+def test_zero_budget_keeps_only_the_shared_experts(S, T):
+    """K_base = 0 and budget = 0: no routed pair is kept (Sec. 4's K_base ablation allows tokens without a routed
+    expert); the output is the shared experts' alone, or zero.  The same through the routed entry with n_sel = 0."""
+    cfg = synth.MoEConfig("zero", T=T, H=128, N=8, I=128, S=S, K_orig=2, K_base=0, budget=0, seed=5)
+    d = dev_layer(cfg)
+    out, inter, status = forward_gpu(cfg, d, 0)
+    assert status == 0
+    assert int(inter["n_sel"].sum()) == 0 and int(inter["expert_offsets"][-1]) == 0
+    assert (inter["pair_pos"] == -1).all()
+    want = orc.shared_experts(np32(d["x"]), np32(d["Wsh13"]), np32(d["Wsh2"])) if S else np.zeros((T, cfg.H))
+    got = out.float().cpu().numpy()
+    if S:
+        assert max_rel(got, want) <= TOL_OUT
+    else:
+        assert (got == 0).all()
+    shape = B.shape_of(cfg)
+    for bmax in (0, 10):
+        ws = B.new_workspace(shape, bmax)
+        out2 = torch.full_like(d["x"], 9.0)
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        B.moe_layer_forward_routed(shape, d["x"], inter["topk_idx"], inter["topk_score"], inter["n_sel"], bmax, 0, d["W13"],
+                                   d["W2"], d["Wsh13"], d["Wsh2"], out2, st, ws)
+        torch.cuda.synchronize()
+        assert st.item() == 0 and torch.equal(out2, out)
+
+
 def test_residual_flag_adds_the_input():
     cfg = synth.CONFIGS["c1k0"]
     d = dev_layer(cfg)
